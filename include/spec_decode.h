@@ -1,0 +1,182 @@
+/*
+ * spec_decode.h -- C ABI of the draft-and-verify decode loop (Sec. III-B of
+ * "Speculative Decoding for Verilog: Speed and Quality, All in One").
+ *
+ * One decode step, as the paper states it: with the model at position t the base model
+ * predicts the token at t+1 and extra head i predicts the token at t+i+1; the heads'
+ * top-k predictions form several candidates; the base model scores every candidate
+ * position; a token is accepted only if the acceptance rule holds for it and for every
+ * token before it; the step emits the longest accepted prefix among all candidates.
+ *
+ * Conventions
+ *  - All functions return 0 on success or a negative SPEC_E_* code. Nothing aborts,
+ *    throws or traps; spec_last_error() gives a one-line description of the last failure.
+ *  - "DEVICE" pointers are CUDA global memory of the device that was current at
+ *    spec_create. "HOST" pointers are ordinary (preferably pinned) host memory.
+ *  - The library never allocates or frees device memory. The caller owns weights,
+ *    workspace and the stream; they must outlive the context.
+ *  - Linear weights are row-major [out_features, in_features]; dtype 0 = float32,
+ *    dtype 1 = bfloat16 (operands bf16, accumulation and residual stream float32).
+ */
+#ifndef SPEC_DECODE_H_
+#define SPEC_DECODE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPEC_MAX_NODES 128   /* tree nodes per sequence, root included          */
+#define SPEC_MAX_HEADS 16    /* extra decoding heads                            */
+#define SPEC_MAX_TOPK 16     /* candidates kept per head                        */
+
+enum {
+  SPEC_OK = 0,
+  SPEC_E_BADARG = -1,   /* null pointer, non-positive size, unsupported shape            */
+  SPEC_E_BADTREE = -2,  /* tree violates the rules listed at spec_tree                    */
+  SPEC_E_NOMEM = -3,    /* workspace too small                                            */
+  SPEC_E_SEQLEN = -4,   /* a sequence would exceed max_seq                                */
+  SPEC_E_CUDA = -5,     /* a CUDA runtime or driver call failed                           */
+  SPEC_E_TIMEOUT = -6,  /* a bounded device-side wait expired (device status word)        */
+  SPEC_E_STATE = -7     /* call out of order (step before prefill, batch mismatch)        */
+};
+
+typedef struct spec_ctx spec_ctx; /* opaque */
+
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rms_eps, rope_base;
+  int32_t dtype;        /* 0 = float32, 1 = bfloat16                                      */
+  int32_t n_medusa;     /* K extra heads (Sec. III-B)                                      */
+  int32_t max_batch;    /* sequences decoded together                                     */
+  int32_t max_seq;      /* committed tokens per sequence (prompt + generated)             */
+  int32_t page_size;    /* tokens per KV page (16)                                        */
+  int32_t accept_mode;  /* 0 = greedy argmax match; 1 = typical acceptance (Eq. 1)        */
+  float typ_eps, typ_delta, temperature; /* Eq. 1 hyper-parameters; softmax temperature   */
+  int32_t frag_token;   /* fragment marker id for the fragment-integrity rule; -1 = off   */
+  int32_t flags;        /* SPEC_FLAG_* bits                                               */
+} spec_config;
+
+#define SPEC_FLAG_KEEP_LOGITS 1 /* materialise verify logits [rows, vocab] for spec_debug_read  */
+#define SPEC_FLAG_SIMPLE_KERNELS 2 /* bf16: run the plain CUDA-core kernels (debug aid, slow)  */
+
+/* Candidate tree, HOST arrays of n_nodes entries, copied at spec_create. Rules: node 0 is
+ * the root (parent -1, depth 0, rank 0) and carries the base model's own next token;
+ * parent[v] < v; depth[v] = depth[parent[v]] + 1 <= n_medusa; node v carries candidate
+ * rank[v] (< SPEC_MAX_TOPK) of head depth[v]; siblings have distinct ranks;
+ * 1 <= n_nodes <= SPEC_MAX_NODES. */
+typedef struct {
+  int32_t n_nodes;
+  const int32_t *parent, *depth, *rank;
+} spec_tree;
+
+/* DEVICE pointers to the weights (HOST arrays of DEVICE pointers where indexed by layer or
+ * head). Element type follows spec_config.dtype except the RMSNorm gains, which are
+ * always float32. */
+typedef struct {
+  const void *embed;            /* [vocab, d_model]                                      */
+  const void *lm_head;          /* [vocab, d_model], untied                              */
+  const float *final_norm;      /* [d_model]                                             */
+  const float *const *attn_norm; /* [n_layers] -> [d_model]                              */
+  const void *const *wq;        /* [n_layers] -> [n_heads*head_dim, d_model]             */
+  const void *const *wk;        /* [n_layers] -> [n_kv_heads*head_dim, d_model]          */
+  const void *const *wv;        /* [n_layers] -> [n_kv_heads*head_dim, d_model]          */
+  const void *const *wo;        /* [n_layers] -> [d_model, n_heads*head_dim]             */
+  const float *const *ffn_norm; /* [n_layers] -> [d_model]                               */
+  const void *const *w_gate;    /* [n_layers] -> [d_ffn, d_model]                        */
+  const void *const *w_up;      /* [n_layers] -> [d_ffn, d_model]                        */
+  const void *const *w_down;    /* [n_layers] -> [d_model, d_ffn]                        */
+  const void *const *medusa_w;  /* [n_medusa] -> [d_model, d_model]                      */
+  const void *const *medusa_b;  /* [n_medusa] -> [d_model]                               */
+} spec_weights;
+
+/* Bytes of DEVICE workspace spec_create needs for this shape and tree (KV page pool, page
+ * tables, activations, split-K and split-KV scratch, status word). 0 on invalid input. */
+size_t spec_workspace_bytes(const spec_config *cfg, const spec_tree *tree);
+
+/* Builds a context. `workspace` is a DEVICE buffer of at least spec_workspace_bytes(),
+ * 1024-byte aligned, zero-filled or not (the library initialises what it needs).
+ * `cuda_stream` is a cudaStream_t (NULL = default stream); all work is enqueued on it.
+ * If the q/k/v matrices of a layer are one contiguous allocation in the order wq, wk, wv
+ * (wk[l] == wq[l] + n_heads*head_dim*d_model elements, and so on) the three projections
+ * run as one launch; otherwise as three.
+ * Config and tree are copied; weights, workspace and stream are borrowed. */
+int spec_create(const spec_config *cfg, const spec_weights *weights, const spec_tree *tree,
+                void *workspace, size_t workspace_bytes, void *cuda_stream, spec_ctx **out);
+
+/* Prompt processing: causal forward over `batch` prompts (HOST token ids, concatenated;
+ * offsets[batch+1] HOST). Fills the KV cache for positions 0..len-1 of every sequence,
+ * keeps each sequence's last hidden state for the first step's heads and sets the first
+ * root token to the base model's argmax at the last prompt position. Resets any earlier
+ * decode state. Synchronous. */
+int spec_prefill(spec_ctx *ctx, int32_t batch, const int32_t *tokens, const int32_t *offsets);
+
+/* One draft-and-verify step for every sequence of the batch (Sec. III-B):
+ *  heads + shared lm_head + per-head top-k -> candidate tree -> one tree-masked
+ *  verification forward of the base model -> longest accepted prefix (greedy: a node is
+ *  accepted iff its token is the base model's argmax at its parent and its parent is
+ *  accepted; ties between equally long paths go to the lowest node index) -> the accepted
+ *  path's K/V rows are moved to the next cache positions.
+ * out_tokens [batch][n_medusa+1] and out_counts [batch] are HOST buffers: sequence b emitted
+ * out_counts[b] in [1, n_medusa+1] tokens, the accepted path root first. The call returns
+ * after they are valid. If both are NULL the step is only enqueued on the stream (no host
+ * synchronisation); emitted tokens are then read later with spec_read_generated.
+ * cand_override: optional HOST table [batch][n_medusa][kmax] (kmax = spec_query(SPEC_Q_KMAX));
+ * an entry >= 0 replaces that head candidate after the heads have run, -1 keeps it. */
+int spec_step(spec_ctx *ctx, int32_t *out_tokens, int32_t *out_counts, const int32_t *cand_override);
+
+/* Copies up to `max_tokens` tokens generated so far by sequence `seq` (all steps since
+ * prefill, in order) to HOST `out` and the total count to *n_generated. Synchronises. */
+int spec_read_generated(spec_ctx *ctx, int32_t seq, int32_t *out, int32_t max_tokens, int32_t *n_generated);
+
+int spec_destroy(spec_ctx *ctx);
+
+/* Description of the last error of this context (or of the last failed spec_create when
+ * ctx is NULL). Never NULL. */
+const char *spec_last_error(const spec_ctx *ctx);
+
+/* Integer properties of a context. */
+enum { SPEC_Q_KMAX = 0, SPEC_Q_KERNEL_LAUNCHES = 1, SPEC_Q_N_NODES = 2, SPEC_Q_BATCH = 3,
+       SPEC_Q_ALGO_BYTES_PER_STEP = 4 /* weights + lm_head (twice) + heads, in KiB */ };
+int64_t spec_query(const spec_ctx *ctx, int32_t what);
+
+/* Debug taps (tests): copy an intermediate of the LAST step to HOST memory. Synchronises.
+ * Rows are ordered [sequence][tree node]. */
+enum {
+  SPEC_DBG_TOK = 0,      /* int32 [rows]            tree tokens                               */
+  SPEC_DBG_POS = 1,      /* int32 [rows]            RoPE positions                            */
+  SPEC_DBG_LOGITS = 2,   /* float [rows][vocab]     verify logits (needs SPEC_FLAG_KEEP_LOGITS) */
+  SPEC_DBG_HIDDEN = 3,   /* float [rows][d_model]   hidden state after the final norm        */
+  SPEC_DBG_ARGMAX = 4,   /* int32 [rows]            per-node argmax of the base logits       */
+  SPEC_DBG_PATH = 5,     /* int32 [batch][n_medusa+1] accepted node ids, -1 padded            */
+  SPEC_DBG_CAND = 6,     /* int32 [batch][n_medusa+1][kmax] candidate table                   */
+  SPEC_DBG_SEQLEN = 7,   /* int32 [batch]           committed tokens per sequence             */
+  SPEC_DBG_NEXT_ROOT = 8,/* int32 [batch]           next step's root token                    */
+  SPEC_DBG_H_LAST = 9,   /* float [batch][d_model]  hidden state feeding the next heads       */
+  SPEC_DBG_STATUS = 10   /* int32 [4]               device status word (0 = clean)            */
+};
+int spec_debug_read(spec_ctx *ctx, int32_t what, void *host_buf, size_t bytes);
+
+/* Copies cached K and V rows of sequence `seq`, layer `layer`, slots [slot0, slot0+n_slots)
+ * to HOST float32 arrays [n_slots][n_kv_heads][head_dim] in logical (unpaged) order. */
+int spec_debug_read_kv(spec_ctx *ctx, int32_t seq, int32_t layer, int32_t slot0, int32_t n_slots,
+                       float *host_k, float *host_v);
+
+/* ---- single operations of the verify forward, for unit parity tests and profiling ---- */
+
+/* y[M,N] (float32, DEVICE) = x[M,K] * W[N,K]^T for DEVICE x and W of type `dtype`
+ * (Sec. III-B verification forward: every projection of the base model). bf16 runs the
+ * tensor-core weight-streaming kernel with `splits` K-slices whose float32 partial sums
+ * are written to `scratch` (DEVICE, splits*M*N + 4 floats; the last four hold the call's
+ * status word) and then summed into y in slice order; float32 runs the CUDA-core row kernel
+ * (splits and scratch ignored). M <= 2048; for bf16 K % 64 == 0 and M % 16 == 0.
+ * Synchronises in bf16 mode. */
+int spec_op_linear(int32_t dtype, const void *x, const void *w, float *y, int32_t M, int32_t N,
+                   int32_t K, int32_t splits, float *scratch, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPEC_DECODE_H_ */

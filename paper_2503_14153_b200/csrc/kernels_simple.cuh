@@ -1,0 +1,625 @@
+// CUDA-core kernels of the decode step: row preparation, RMSNorm, row-streaming linear
+// (the float32 path and the M<=few GEMV-style projections of the extra heads), RoPE + cache
+// store, plain tree attention, argmax, acceptance walk, KV compaction, per-head top-k.
+// Templated on the operand type T (float or bf16): operands are rounded to T exactly where
+// a tensor-core kernel would consume them; accumulation is float32.
+#pragma once
+#include "common.cuh"
+
+namespace spec {
+
+// Per-pass row bookkeeping. Row m = b * R + i belongs to sequence b; it is valid iff
+// i < cnt[b]. n[b] cached positions precede the pass's rows of sequence b.
+struct Rows {
+  int R, B;
+  int *tok, *pos, *slot;  // [B*R]
+  int *n, *cnt;           // [B]
+  const uint32_t* anc;    // [R][4] ancestor bitsets (bit u of anc[i]: row i sees row u)
+};
+
+// ------------------------------------------------------------------ row preparation
+// Verify pass: tree node i of sequence b carries candidate rank[i] of head depth[i]
+// (head 0 = the base model's own next token) and sits at position n[b] + depth[i].
+template <typename T>
+__global__ void prepare_verify_rows(Rows rows, const int* __restrict__ cand, int cand_stride_b, int kmax,
+                                    const int* __restrict__ depth, const int* __restrict__ rank, int capacity,
+                                    const T* __restrict__ embed, float* __restrict__ x, int d, int vocab,
+                                    int* status) {
+  int m = blockIdx.x, b = m / rows.R, i = m % rows.R;
+  int n = rows.n[b];
+  bool ok = (n + rows.R <= capacity);
+  if (!ok && threadIdx.x == 0) set_status(status, ST_SEQLEN, 1, b);
+  int t = cand[b * cand_stride_b + depth[i] * kmax + rank[i]];
+  if (t < 0 || t >= vocab) { t = 0; if (threadIdx.x == 0 && ok) set_status(status, ST_BOUNDS, 1, m); }
+  if (threadIdx.x == 0) {
+    rows.tok[m] = t;
+    rows.pos[m] = n + depth[i];
+    rows.slot[m] = n + i;
+    if (i == 0) rows.cnt[b] = ok ? rows.R : 0;
+  }
+  const T* e = embed + (size_t)t * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)m * d + c] = to_f<T>(e[c]);
+}
+
+// Prefill pass number `chunk`: row i of sequence b is prompt token chunk*R + i.
+template <typename T>
+__global__ void prepare_prefill_rows(Rows rows, const int* __restrict__ prompt, const int* __restrict__ offsets,
+                                     int chunk, const T* __restrict__ embed, float* __restrict__ x, int d,
+                                     int vocab, int* status) {
+  int m = blockIdx.x, b = m / rows.R, i = m % rows.R;
+  int len = offsets[b + 1] - offsets[b];
+  int p = chunk * rows.R + i;
+  int t = 0;
+  if (p < len) {
+    t = prompt[offsets[b] + p];
+    if (t < 0 || t >= vocab) { t = 0; if (threadIdx.x == 0) set_status(status, ST_BOUNDS, 2, m); }
+  }
+  if (threadIdx.x == 0) {
+    rows.tok[m] = t;
+    rows.pos[m] = p;
+    rows.slot[m] = p;
+    if (i == 0) {
+      int c = len - chunk * rows.R;
+      rows.cnt[b] = c < 0 ? 0 : (c > rows.R ? rows.R : c);
+      rows.n[b] = chunk * rows.R < len ? chunk * rows.R : len;
+    }
+  }
+  const T* e = embed + (size_t)t * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)m * d + c] = (p < len) ? to_f<T>(e[c]) : 0.f;
+}
+
+// After a prefill pass: sequences whose last prompt token is in this pass keep that row's
+// final hidden state (float32 and operand type) for the first step's heads and lm_head.
+template <typename T>
+__global__ void prefill_keep_last(Rows rows, const int* __restrict__ offsets, int chunk,
+                                  const float* __restrict__ hid, float* __restrict__ h_last,
+                                  T* __restrict__ hq_last, int d) {
+  int b = blockIdx.x;
+  int len = offsets[b + 1] - offsets[b];
+  int last = len - 1;
+  if (last / rows.R != chunk) return;
+  int m = b * rows.R + last % rows.R;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float v = hid[(size_t)m * d + c];
+    h_last[(size_t)b * d + c] = v;
+    hq_last[(size_t)b * d + c] = from_f<T>(v);
+  }
+  if (threadIdx.x == 0) rows.n[b] = len;
+}
+
+// ------------------------------------------------------------------ RMSNorm (+ residual)
+// x[m] += sum_s part[s][m] (s in slice order) when nsplit > 0; u[m] = T(x / rms(x) * g);
+// optionally the unrounded normed row goes to hid (final norm).
+template <typename T>
+__global__ void rmsnorm_rows(float* __restrict__ x, const float* __restrict__ part, int nsplit, size_t split_stride,
+                             const float* __restrict__ gain, float eps, T* __restrict__ u,
+                             float* __restrict__ hid, int d) {
+  int m = blockIdx.x;
+  float* xr = x + (size_t)m * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float v = xr[c];
+    for (int s = 0; s < nsplit; ++s) v += part[s * split_stride + (size_t)m * d + c];
+    if (nsplit > 0) xr[c] = v;
+    ss += v * v;
+  }
+  __shared__ float red[32];
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+    v = warp_sum(v);
+    if (threadIdx.x == 0) red[0] = v;
+  }
+  __syncthreads();
+  float inv = rsqrtf(red[0] / (float)d + eps);
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float v = xr[c] * inv * gain[c];
+    u[(size_t)m * d + c] = from_f<T>(v);
+    if (hid) hid[(size_t)m * d + c] = v;
+  }
+}
+
+// ------------------------------------------------------------------ row-streaming linear
+// y[m][n] = sum_k x[m][k] * W[n][k] for MC rows m at a time; one warp per output n streams
+// the weight row once with 16-byte loads. K % 8 == 0.
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+  static constexpr int N = 4;
+  __device__ static void load(const float* p, float (&o)[8]) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+  }
+};
+template <> struct Vec16<bf16> {
+  static constexpr int N = 8;
+  __device__ static void load(const bf16* p, float (&o)[8]) {
+    uint4 v = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { float2 f = __bfloat1622float2(h[i]); o[2 * i] = f.x; o[2 * i + 1] = f.y; }
+  }
+};
+
+template <typename T, int MC>
+__global__ void linear_rows(const T* __restrict__ x, int ldx, const T* __restrict__ W, float* __restrict__ y,
+                            int ldy, int M, int N, int K) {
+  constexpr int VN = Vec16<T>::N;
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int n = blockIdx.x * (blockDim.x >> 5) + warp;
+  int m0 = blockIdx.y * MC;
+  if (n >= N) return;
+  float acc[MC];
+#pragma unroll
+  for (int i = 0; i < MC; ++i) acc[i] = 0.f;
+  const T* wr = W + (size_t)n * K;
+  for (int k = lane * VN; k < K; k += 32 * VN) {
+    float wv[8], xv[8];
+    Vec16<T>::load(wr + k, wv);
+#pragma unroll
+    for (int i = 0; i < MC; ++i) {
+      if (m0 + i < M) {
+        Vec16<T>::load(x + (size_t)(m0 + i) * ldx + k, xv);
+#pragma unroll
+        for (int e = 0; e < VN; ++e) acc[i] = fmaf(wv[e], xv[e], acc[i]);
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < MC; ++i) {
+    float v = warp_sum(acc[i]);
+    if (lane == 0 && m0 + i < M) y[(size_t)(m0 + i) * ldy + n] = v;
+  }
+}
+
+// y = sum over K slices, in slice order
+__global__ void sum_partials(const float* __restrict__ part, int nsplit, size_t total, float* __restrict__ y) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  float v = 0.f;
+  for (int s = 0; s < nsplit; ++s) v += part[(size_t)s * total + i];
+  y[i] = v;
+}
+
+// act = T(SiLU(g) * u)
+template <typename T>
+__global__ void swiglu_rows(const float* __restrict__ g, const float* __restrict__ up, T* __restrict__ act,
+                            size_t total) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < total) act[i] = from_f<T>(silu_f(g[i]) * up[i]);
+}
+
+// ------------------------------------------------------------------ RoPE + cache store
+// qkv: float32 [nsplit][M][(H+2Hkv)*D] partial sums. Rotate-half RoPE (element i pairs with
+// i + D/2, angle pos * base^(-2i/D), table cs[pos][i] = (cos, sin)) on q and k; q -> T
+// [M][H*D]; k, v -> T into the paged cache at the row's slot.
+template <typename T>
+__global__ void rope_store(const float* __restrict__ qkv, int nsplit, size_t split_stride, Rows rows,
+                           const float2* __restrict__ cs, T* __restrict__ q, T* __restrict__ pool, KVGeom g,
+                           const int* __restrict__ page_table, int layer, int H) {
+  int m = blockIdx.x, b = m / rows.R, i = m % rows.R;
+  if (i >= rows.cnt[b]) return;
+  int D = g.head_dim, half = D >> 1, Hkv = g.n_kv_heads;
+  int nq = H * D, nk = Hkv * D, ld = nq + 2 * nk;
+  int pos = rows.pos[m], slot = rows.slot[m];
+  int page = page_table[b * g.pages_per_seq + slot / g.page_size], prow = slot % g.page_size;
+  const float* src = qkv + (size_t)m * ld;
+  // q and k pairs
+  int npairs = (H + Hkv) * half;
+  for (int p = threadIdx.x; p < npairs; p += blockDim.x) {
+    int head = p / half, e = p % half;
+    int col = head * D + e;
+    float a = 0.f, c = 0.f;
+    for (int s = 0; s < max(nsplit, 1); ++s) {
+      a += src[s * split_stride + col];
+      c += src[s * split_stride + col + half];
+    }
+    float2 t = cs[(size_t)pos * half + e];
+    float r0 = a * t.x - c * t.y, r1 = c * t.x + a * t.y;
+    if (head < H) {
+      q[(size_t)m * nq + head * D + e] = from_f<T>(r0);
+      q[(size_t)m * nq + head * D + e + half] = from_f<T>(r1);
+    } else {
+      int kh = head - H;
+      T* dst = pool + g.block_offset(page, layer, 0, kh) + (size_t)prow * D;
+      dst[kv_elem<T>(prow, e)] = from_f<T>(r0);
+      dst[kv_elem<T>(prow, e + half)] = from_f<T>(r1);
+    }
+  }
+  for (int p = threadIdx.x; p < nk; p += blockDim.x) {
+    int kh = p / D, e = p % D;
+    float a = 0.f;
+    for (int s = 0; s < max(nsplit, 1); ++s) a += src[s * split_stride + nq + nk + p];
+    T* dst = pool + g.block_offset(page, layer, 1, kh) + (size_t)prow * D;
+    dst[kv_elem<T>(prow, e)] = from_f<T>(a);
+  }
+}
+
+// ------------------------------------------------------------------ plain tree attention
+// One warp per (row, head). Row i of sequence b sees every cached position < n[b] and row u
+// of the same pass iff bit u of anc[i] is set. Two passes over the keys: maximum, then
+// exp / sum / value accumulation with the probabilities rounded to T before the product.
+template <typename T>
+__global__ void attention_simple(const T* __restrict__ q, T* __restrict__ out, const T* __restrict__ pool, KVGeom g,
+                                 const int* __restrict__ page_table, Rows rows, int layer, int H, float scale) {
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int h = blockIdx.x, b = blockIdx.y;
+  int i = blockIdx.z * (blockDim.x >> 5) + warp;
+  if (i >= rows.cnt[b]) return;
+  int m = b * rows.R + i;
+  int D = g.head_dim, EPL = D >> 5;   // D in {32,64,128,256}
+  int kvh = h / (H / g.n_kv_heads);
+  int n = rows.n[b], S = n + rows.cnt[b];
+  float qv[8];
+  for (int e = 0; e < EPL; ++e) qv[e] = to_f<T>(q[(size_t)m * H * D + h * D + lane * EPL + e]);
+  uint32_t a[4];
+  for (int w = 0; w < 4; ++w) a[w] = rows.anc[i * 4 + w];
+  const int* pt = page_table + b * g.pages_per_seq;
+
+  float mx = -INFINITY;
+  for (int j = 0; j < S; ++j) {
+    if (j >= n && !((a[(j - n) >> 5] >> ((j - n) & 31)) & 1u)) continue;
+    int prow = j % g.page_size;
+    const T* kr = pool + g.block_offset(pt[j / g.page_size], layer, 0, kvh) + (size_t)prow * D;
+    float s = 0.f;
+    for (int e = 0; e < EPL; ++e) s = fmaf(qv[e], to_f<T>(kr[kv_elem<T>(prow, lane * EPL + e)]), s);
+    s = warp_sum(s) * scale;
+    mx = fmaxf(mx, s);
+  }
+  float l = 0.f, acc[8];
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  for (int j = 0; j < S; ++j) {
+    if (j >= n && !((a[(j - n) >> 5] >> ((j - n) & 31)) & 1u)) continue;
+    int prow = j % g.page_size;
+    int page = pt[j / g.page_size];
+    const T* kr = pool + g.block_offset(page, layer, 0, kvh) + (size_t)prow * D;
+    const T* vr = pool + g.block_offset(page, layer, 1, kvh) + (size_t)prow * D;
+    float s = 0.f;
+    for (int e = 0; e < EPL; ++e) s = fmaf(qv[e], to_f<T>(kr[kv_elem<T>(prow, lane * EPL + e)]), s);
+    s = warp_sum(s) * scale;
+    float p = expf(s - mx);
+    l += p;
+    float pq = quant<T>(p);
+    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pq, to_f<T>(vr[kv_elem<T>(prow, lane * EPL + e)]), acc[e]);
+  }
+  float inv = 1.f / l;
+  for (int e = 0; e < EPL; ++e) out[(size_t)m * H * D + h * D + lane * EPL + e] = from_f<T>(acc[e] * inv);
+}
+
+// ------------------------------------------------------------------ argmax over vocabulary
+// One block per row; lowest index wins ties. Writes one (value, index) partial per row.
+__global__ void argmax_rows(const float* __restrict__ logits, int V, float* __restrict__ pval, int* __restrict__ pidx) {
+  int m = blockIdx.x;
+  const float* z = logits + (size_t)m * V;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) {
+    float v = z[c];
+    if (better(v, c, bv, bi)) { bv = v; bi = c; }
+  }
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  warp_argmax(bv, bi);
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    int nw = blockDim.x >> 5;
+    bv = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
+    bi = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
+    warp_argmax(bv, bi);
+    if (threadIdx.x == 0) { pval[m] = bv; pidx[m] = bi; }
+  }
+}
+
+// ------------------------------------------------------------------ typical acceptance
+// Eq. 1: a node passes iff p_base(token | prefix ending at its parent) >
+// min(eps, delta * exp(-H(p_base))). One block per node v; it reduces its parent's logits
+// row (softmax at the given temperature, entropy in nats).
+__global__ void typical_edges(const float* __restrict__ logits, int V, Rows rows, const int* __restrict__ parent,
+                              float eps, float delta, float inv_temp, int* __restrict__ edge_ok) {
+  int m = blockIdx.x, b = m / rows.R, v = m % rows.R;
+  if (v >= rows.cnt[b]) return;
+  if (v == 0) { if (threadIdx.x == 0) edge_ok[m] = 1; return; }
+  const float* z = logits + (size_t)(b * rows.R + parent[v]) * V;
+  __shared__ float red[32];
+  __shared__ float bc[2];
+  float mx = -INFINITY;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) mx = fmaxf(mx, z[c] * inv_temp);
+  mx = warp_max(mx);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float t = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : -INFINITY;
+    t = warp_max(t);
+    if (threadIdx.x == 0) bc[0] = t;
+  }
+  __syncthreads();
+  mx = bc[0];
+  float se = 0.f, sez = 0.f;   // sum e, sum e * (z - mx)
+  for (int c = threadIdx.x; c < V; c += blockDim.x) {
+    float t = z[c] * inv_temp - mx;
+    float e = expf(t);
+    se += e;
+    sez += e * t;
+  }
+  se = warp_sum(se);
+  sez = warp_sum(sez);
+  __shared__ float red2[32];
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = se; red2[threadIdx.x >> 5] = sez; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    int nw = blockDim.x >> 5;
+    float a = threadIdx.x < nw ? red[threadIdx.x] : 0.f, c = threadIdx.x < nw ? red2[threadIdx.x] : 0.f;
+    a = warp_sum(a);
+    c = warp_sum(c);
+    if (threadIdx.x == 0) {
+      float H = logf(a) - c / a;                 // -sum p log p with p = e / a
+      float thr = fminf(eps, delta * expf(-H));
+      float p = expf(z[rows.tok[m]] * inv_temp - mx) / a;
+      edge_ok[m] = p > thr ? 1 : 0;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ acceptance walk
+struct AcceptArgs {
+  Rows rows;
+  const float* pval;   // [ntile][pstride]
+  const int* pidx;
+  int ntile, pstride;
+  const int *parent, *depth;   // tree arrays [R]
+  const int* edge_ok;          // typical mode: per-row pass flag; NULL = greedy token match
+  int K, frag_token, d, mode;  // mode 0 = verify step, 1 = prefill (row b is sequence b)
+  const float* hid;            // [rows][d]
+  int *am, *path, *count, *out_tok, *n_old, *root_tok;
+  float* h_last;
+  int *gen_log, *gen_cnt, gen_cap;
+};
+
+// One block per sequence: finishes the per-node argmax from the per-tile partials, walks the
+// tree (a node is accepted iff its parent is and its token is the argmax at the parent, or
+// its Eq. 1 flag is set), takes the deepest accepted node (lowest index on ties), applies
+// the fragment-integrity rule, and publishes the step's result and the next step's state.
+__global__ void accept_kernel(AcceptArgs a) {
+  int b = blockIdx.x, R = a.rows.R;
+  __shared__ int am_s[SPEC_MAX_NODES];
+  __shared__ int last_s, len_s;
+  if (a.mode == 1) {
+    if (threadIdx.x == 0) {
+      float bv = -INFINITY; int bi = 0x7fffffff;
+      for (int t = 0; t < a.ntile; ++t) {
+        float v = a.pval[(size_t)t * a.pstride + b]; int i = a.pidx[(size_t)t * a.pstride + b];
+        if (better(v, i, bv, bi)) { bv = v; bi = i; }
+      }
+      a.am[b] = bi;
+      a.root_tok[b] = bi;
+      a.gen_cnt[b] = 0;
+    }
+    return;
+  }
+  int cnt = a.rows.cnt[b], m0 = b * R;
+  for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+    float bv = -INFINITY; int bi = 0x7fffffff;
+    for (int t = 0; t < a.ntile; ++t) {
+      float v = a.pval[(size_t)t * a.pstride + m0 + i]; int idx = a.pidx[(size_t)t * a.pstride + m0 + i];
+      if (better(v, idx, bv, bi)) { bv = v; bi = idx; }
+    }
+    am_s[i] = bi;
+    a.am[m0 + i] = bi;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int len = 0, last = 0;
+    for (int j = 0; j <= a.K; ++j) a.path[b * (a.K + 1) + j] = -1;
+    if (cnt > 0) {
+      // acc bits in registers: up to 128 nodes
+      uint32_t acc[4] = {1u, 0u, 0u, 0u};
+      int best = 0;
+      for (int v = 1; v < cnt; ++v) {
+        int p = a.parent[v];
+        bool ok = (acc[p >> 5] >> (p & 31)) & 1u;
+        if (ok) ok = a.edge_ok ? (a.edge_ok[m0 + v] != 0) : (a.rows.tok[m0 + v] == am_s[p]);
+        if (ok) {
+          acc[v >> 5] |= 1u << (v & 31);
+          if (a.depth[v] > a.depth[best]) best = v;
+        }
+      }
+      len = a.depth[best] + 1;
+      int path[SPEC_MAX_HEADS + 1];
+      for (int u = best; u >= 0; u = a.parent[u]) path[a.depth[u]] = u;
+      if (a.frag_token >= 0) {
+        int keep = 1;
+        for (int j = 0; j < len; ++j) if (a.rows.tok[m0 + path[j]] == a.frag_token) keep = j + 1;
+        len = keep;
+      }
+      int n = a.rows.n[b], gc = a.gen_cnt[b];
+      for (int j = 0; j < len; ++j) {
+        int t = a.rows.tok[m0 + path[j]];
+        a.path[b * (a.K + 1) + j] = path[j];
+        a.out_tok[b * (a.K + 1) + j] = t;
+        if (gc + j < a.gen_cap) a.gen_log[(size_t)b * a.gen_cap + gc + j] = t;
+      }
+      last = path[len - 1];
+      a.n_old[b] = n;
+      a.rows.n[b] = n + len;
+      a.gen_cnt[b] = gc + len;
+      a.root_tok[b] = am_s[last];
+    }
+    a.count[b] = len;
+    last_s = last; len_s = len;
+  }
+  __syncthreads();
+  if (len_s > 0) {
+    const float* src = a.hid + (size_t)(m0 + last_s) * a.d;
+    for (int c = threadIdx.x; c < a.d; c += blockDim.x) a.h_last[(size_t)b * a.d + c] = src[c];
+  }
+}
+
+// ------------------------------------------------------------------ KV compaction
+// Moves the accepted path's K/V rows from slot n_old + path[j] to slot n_old + j, for every
+// layer and KV head. path[j] >= j and strictly increasing, so processing j in ascending
+// order by the same thread never overwrites a row that is still to be read.
+template <typename T>
+__global__ void compact_kv(T* __restrict__ pool, KVGeom g, const int* __restrict__ page_table,
+                           const int* __restrict__ path, const int* __restrict__ count,
+                           const int* __restrict__ n_old, int K) {
+  int b = blockIdx.y;
+  int blk = blockIdx.x;              // (layer*2 + kv) * Hkv + head
+  int head = blk % g.n_kv_heads, lk = blk / g.n_kv_heads;
+  int len = count[b];
+  int D = g.head_dim;
+  const int* pt = page_table + b * g.pages_per_seq;
+  int n0 = n_old[b];
+  for (int j = 0; j < len; ++j) {
+    int src = n0 + path[b * (K + 1) + j], dst = n0 + j;
+    if (src == dst) continue;
+    int sr = src % g.page_size, dr = dst % g.page_size;
+    const T* s = pool + g.block_offset(pt[src / g.page_size], lk >> 1, lk & 1, head) + (size_t)sr * D;
+    T* t = pool + g.block_offset(pt[dst / g.page_size], lk >> 1, lk & 1, head) + (size_t)dr * D;
+    for (int e = threadIdx.x; e < D; e += blockDim.x) t[kv_elem<T>(dr, e)] = s[kv_elem<T>(sr, e)];
+  }
+}
+
+// ------------------------------------------------------------------ extra decoding heads
+// r[b][k] = T(h + SiLU(W_k h + b_k)), h = T(h_last[b]). One warp per output element row i of
+// head k; MC sequences at a time.
+template <typename T, int MC>
+__global__ void medusa_resblock(const float* __restrict__ h_last, const T* const* __restrict__ Wk,
+                                const T* const* __restrict__ bk, T* __restrict__ r, int B, int K, int d) {
+  constexpr int VN = Vec16<T>::N;
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int row = blockIdx.x * (blockDim.x >> 5) + warp;   // k * d + i
+  int b0 = blockIdx.y * MC;
+  if (row >= K * d) return;
+  int k = row / d, i = row % d;
+  const T* wr = Wk[k] + (size_t)i * d;
+  float acc[MC];
+#pragma unroll
+  for (int j = 0; j < MC; ++j) acc[j] = 0.f;
+  for (int c = lane * VN; c < d; c += 32 * VN) {
+    float wv[8];
+    Vec16<T>::load(wr + c, wv);
+#pragma unroll
+    for (int j = 0; j < MC; ++j) {
+      if (b0 + j < B) {
+        const float* hr = h_last + (size_t)(b0 + j) * d + c;
+#pragma unroll
+        for (int e = 0; e < VN; ++e) acc[j] = fmaf(wv[e], quant<T>(hr[e]), acc[j]);
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < MC; ++j) {
+    float v = warp_sum(acc[j]);
+    if (lane == 0 && b0 + j < B) {
+      float h = quant<T>(h_last[(size_t)(b0 + j) * d + i]);
+      r[((size_t)(b0 + j) * K + k) * d + i] = from_f<T>(h + silu_f(v + to_f<T>(bk[k][i])));
+    }
+  }
+}
+
+// z[row][n] = W_lm[n] . r[row] for MC rows (row = b*K + k) over this block's slice of the
+// vocabulary, kept in shared memory; then each row's kmax best (value desc, index asc) of
+// the slice go to the partial lists pk_val/pk_idx [block][rows][kmax].
+template <typename T, int MC>
+__global__ void medusa_lmhead_topk(const T* __restrict__ r, const T* __restrict__ Wlm, int rows_total, int V, int d,
+                                   int slice, int kmax, float* __restrict__ pk_val, int* __restrict__ pk_idx) {
+  constexpr int VN = Vec16<T>::N;
+  extern __shared__ float zs[];   // [MC][slice]
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  int n0 = blockIdx.x * slice, r0 = blockIdx.y * MC;
+  int n1 = min(n0 + slice, V);
+  for (int n = n0 + warp; n < n1; n += nw) {
+    const T* wr = Wlm + (size_t)n * d;
+    float acc[MC];
+#pragma unroll
+    for (int j = 0; j < MC; ++j) acc[j] = 0.f;
+    for (int c = lane * VN; c < d; c += 32 * VN) {
+      float wv[8], xv[8];
+      Vec16<T>::load(wr + c, wv);
+#pragma unroll
+      for (int j = 0; j < MC; ++j) {
+        if (r0 + j < rows_total) {
+          Vec16<T>::load(r + (size_t)(r0 + j) * d + c, xv);
+#pragma unroll
+          for (int e = 0; e < VN; ++e) acc[j] = fmaf(wv[e], xv[e], acc[j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < MC; ++j) {
+      float v = warp_sum(acc[j]);
+      if (lane == 0) zs[j * slice + (n - n0)] = v;
+    }
+  }
+  __syncthreads();
+  for (int j = warp; j < MC; j += nw) {
+    if (r0 + j >= rows_total) continue;
+    float* z = zs + j * slice;
+    for (int t = 0; t < kmax; ++t) {
+      float bv = -INFINITY; int bi = 0x7fffffff;
+      for (int c = lane; c < n1 - n0; c += 32) if (better(z[c], n0 + c, bv, bi)) { bv = z[c]; bi = n0 + c; }
+      warp_argmax(bv, bi);
+      if (lane == 0) {
+        size_t o = ((size_t)blockIdx.x * rows_total + r0 + j) * kmax + t;
+        pk_val[o] = bv;
+        pk_idx[o] = bi;
+        if (bi != 0x7fffffff) z[bi - n0] = -INFINITY;
+      }
+      __syncwarp();
+    }
+  }
+}
+
+// Merges the partial lists of one (sequence, head) row into cand[b][k+1][0..kmax) and applies
+// the optional override table; block 0 of each sequence also writes cand[b][0][0] = root.
+__global__ void topk_merge(const float* __restrict__ pk_val, const int* __restrict__ pk_idx, int nblocks,
+                           int rows_total, int K, int kmax, const int* __restrict__ root_tok,
+                           const int* __restrict__ cand_override, int* __restrict__ cand) {
+  extern __shared__ float ms[];     // values [nblocks*kmax] then indices
+  int row = blockIdx.x, b = row / K, k = row % K;
+  int total = nblocks * kmax;
+  float* v = ms;
+  int* ix = reinterpret_cast<int*>(ms + total);
+  for (int c = threadIdx.x; c < total; c += blockDim.x) {
+    int blk = c / kmax, t = c % kmax;
+    size_t o = ((size_t)blk * rows_total + row) * kmax + t;
+    v[c] = pk_val[o];
+    ix[c] = pk_idx[o];
+  }
+  __syncthreads();
+  __shared__ float sv[32];
+  __shared__ int si[32], sp[32];
+  int* out = cand + ((size_t)b * (K + 1) + k + 1) * kmax;
+  for (int t = 0; t < kmax; ++t) {
+    float bv = -INFINITY; int bi = 0x7fffffff, bp = -1;
+    for (int c = threadIdx.x; c < total; c += blockDim.x)
+      if (better(v[c], ix[c], bv, bi)) { bv = v[c]; bi = ix[c]; bp = c; }
+    // warp then block reduction carrying the position
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, o), op = __shfl_xor_sync(0xffffffffu, bp, o);
+      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bp = op; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; sp[threadIdx.x >> 5] = bp; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 1; w < (blockDim.x >> 5); ++w)
+        if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; bp = sp[w]; }
+      int tokv = bi;
+      if (cand_override) {
+        int o = cand_override[((size_t)b * K + k) * kmax + t];
+        if (o >= 0) tokv = o;
+      }
+      out[t] = (tokv == 0x7fffffff) ? 0 : tokv;
+      if (bp >= 0) v[bp] = -INFINITY, ix[bp] = 0x7fffffff;
+    }
+    __syncthreads();
+  }
+  if (k == 0 && threadIdx.x == 0) cand[(size_t)b * (K + 1) * kmax] = root_tok[b];
+}
+
+}  // namespace spec

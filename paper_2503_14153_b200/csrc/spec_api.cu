@@ -1,0 +1,841 @@
+// C ABI of the draft-and-verify decode loop: context set-up, workspace carving, the
+// per-step kernel schedule and the debug taps. All device work is enqueued on the caller's
+// stream; the library allocates no device memory.
+#include "../../include/spec_decode.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "attention_tc.cuh"
+#include "common.cuh"
+#include "gemm_tc.cuh"
+#include "kernels_simple.cuh"
+
+using namespace spec;
+
+namespace {
+
+thread_local std::string g_create_error = "no error";
+
+constexpr int PREFILL_ROWS = 128;   // rows per sequence in one prefill pass
+constexpr int SM_SLOTS = 296;       // 148 SMs x 2 co-resident GEMM CTAs
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 row-major [rows][cols] matrix, box = box_rows x 64 columns (128 bytes), 128-byte swizzle.
+bool make_tmap(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+struct Bump {
+  uint8_t* base;
+  size_t off = 0;
+  explicit Bump(void* b) : base(static_cast<uint8_t*>(b)) {}
+  template <typename T> T* take(size_t count, size_t align = 256) {
+    off = round_up(off, align);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+int mt_for_rows(int M) {
+  if (M <= 16) return 16;
+  if (M <= 32) return 32;
+  if (M <= 64) return 64;
+  return 128;
+}
+int splits_for(int n_tiles, int m_tiles, int K) {
+  int kc = K / 64;
+  int s = SM_SLOTS / (n_tiles * m_tiles);
+  if (s > 12) s = 12;
+  if (s > kc / 2) s = kc / 2;
+  if (s < 1) s = 1;
+  return s;
+}
+
+}  // namespace
+
+struct spec_ctx {
+  spec_config cfg;
+  cudaStream_t stream;
+  int T, K, kmax, B;                   // tree nodes, heads, candidates per head, current batch
+  bool tc;                             // bf16 tensor-core path
+  size_t esz;                          // operand element size
+  int Mcap, cap, pages_per_seq, gen_cap, nsplit_attn, Nqkv, ntile_lm, topk_slice, topk_blocks;
+  bool qkv_fused, keep_logits;
+  std::vector<int> h_parent, h_depth, h_rank;
+  std::vector<int> n_hi;               // host upper bound of committed lengths
+  std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, mw, mb;
+  std::vector<const float*> an, fn;
+  const void *embed, *lm_head;
+  const float* final_norm;
+  KVGeom geom;
+  // device buffers (workspace)
+  int *d_n, *d_cnt, *d_n_old, *d_root, *d_count, *d_path, *d_out_tok, *d_gen_cnt, *d_gen_log, *d_cand, *d_cand_ov;
+  int *d_tok, *d_pos, *d_slot, *d_am, *d_edge, *d_parent, *d_depth, *d_rank, *d_page_table, *d_prompt, *d_offsets;
+  int *d_status, *d_pidx, *d_pk_idx;
+  uint32_t *d_anc_tree, *d_anc_chain;
+  const void **d_mw, **d_mb;
+  float *d_x, *d_hid, *d_h_last, *d_part, *d_logits, *d_pval, *d_part_o, *d_part_ml, *d_pk_val;
+  float2* d_rope;
+  void *d_u, *d_q, *d_attn, *d_act, *d_hq, *d_hq_last, *d_r, *d_pool;
+  size_t part_floats;
+  std::map<std::tuple<const void*, uint64_t, uint64_t, uint32_t>, CUtensorMap> tmaps;
+  long long launches = 0;
+  bool prefilled = false;
+  std::string err = "no error";
+
+  int fail(int code, const std::string& msg) { err = msg; return code; }
+  const CUtensorMap* tmap(const void* p, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    auto key = std::make_tuple(p, rows, cols, box_rows);
+    auto it = tmaps.find(key);
+    if (it != tmaps.end()) return &it->second;
+    CUtensorMap tm;
+    if (!make_tmap(&tm, p, rows, cols, box_rows)) return nullptr;
+    return &tmaps.emplace(key, tm).first->second;
+  }
+};
+
+namespace {
+
+bool validate_tree(const spec_config* cfg, const spec_tree* tree, int* kmax_out, std::string* why) {
+  int T = tree->n_nodes;
+  if (T < 1 || T > SPEC_MAX_NODES || !tree->parent || !tree->depth || !tree->rank) { *why = "n_nodes out of range or null arrays"; return false; }
+  if (tree->parent[0] != -1 || tree->depth[0] != 0 || tree->rank[0] != 0) { *why = "node 0 must be the root"; return false; }
+  int kmax = 1;
+  for (int v = 1; v < T; ++v) {
+    int p = tree->parent[v];
+    if (p < 0 || p >= v) { *why = "parent must precede child"; return false; }
+    if (tree->depth[v] != tree->depth[p] + 1 || tree->depth[v] > cfg->n_medusa) { *why = "bad depth"; return false; }
+    if (tree->rank[v] < 0 || tree->rank[v] >= SPEC_MAX_TOPK) { *why = "bad rank"; return false; }
+    for (int u = 1; u < v; ++u)
+      if (tree->parent[u] == p && tree->rank[u] == tree->rank[v]) { *why = "siblings share a rank"; return false; }
+    if (tree->rank[v] + 1 > kmax) kmax = tree->rank[v] + 1;
+  }
+  *kmax_out = kmax;
+  return true;
+}
+
+bool validate_config(const spec_config* c, std::string* why) {
+  if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->n_kv_heads < 1 || c->head_dim < 32 ||
+      c->d_ffn < 8 || c->vocab < 2 || c->max_batch < 1 || c->max_seq < 1 || c->page_size < 1) { *why = "non-positive size"; return false; }
+  if (c->dtype != 0 && c->dtype != 1) { *why = "dtype must be 0 or 1"; return false; }
+  if (c->n_heads % c->n_kv_heads) { *why = "n_heads must be a multiple of n_kv_heads"; return false; }
+  if (c->head_dim % 32 || c->head_dim > 256) { *why = "head_dim must be a multiple of 32, <= 256"; return false; }
+  if (c->d_model % 8 || c->d_ffn % 8 || (c->n_heads * c->head_dim) % 8) { *why = "widths must be multiples of 8"; return false; }
+  if (c->n_medusa < 0 || c->n_medusa > SPEC_MAX_HEADS) { *why = "n_medusa out of range"; return false; }
+  if (c->accept_mode != 0 && c->accept_mode != 1) { *why = "accept_mode must be 0 or 1"; return false; }
+  bool tc = c->dtype == 1 && !(c->flags & SPEC_FLAG_SIMPLE_KERNELS);
+  if (tc) {
+    if (c->d_model % 64 || c->d_ffn % 64 || (c->n_heads * c->head_dim) % 64) { *why = "bf16 path needs widths that are multiples of 64"; return false; }
+    if (c->head_dim != 64 && c->head_dim != 128) { *why = "bf16 path needs head_dim 64 or 128"; return false; }
+    if (c->page_size != 16) { *why = "bf16 path needs page_size 16"; return false; }
+  } else if (c->dtype == 1 && c->head_dim % 64) { *why = "bf16 cache needs head_dim multiple of 64"; return false; }
+  return true;
+}
+
+// Lays the workspace out; with base == nullptr only measures it.
+size_t carve(spec_ctx* c, void* base) {
+  const spec_config& f = c->cfg;
+  Bump b(base);
+  int B = f.max_batch, T = c->T, K = c->K, d = f.d_model, F = f.d_ffn, V = f.vocab;
+  int HD = f.n_heads * f.head_dim;
+  c->Nqkv = HD + 2 * f.n_kv_heads * f.head_dim;
+  c->Mcap = (int)round_up((size_t)B * (T > PREFILL_ROWS ? T : PREFILL_ROWS), 128);
+  c->cap = (int)round_up((size_t)f.max_seq + T, f.page_size);
+  if (64 % f.page_size == 0) c->cap = (int)round_up(c->cap, 64);   // whole 64-key attention tiles
+  c->pages_per_seq = c->cap / f.page_size;
+  c->gen_cap = f.max_seq + K + 1;
+  c->ntile_lm = c->tc ? (V + 127) / 128 : 1;
+  c->topk_slice = (V + SM_SLOTS - 1) / SM_SLOTS;
+  c->topk_blocks = (V + c->topk_slice - 1) / c->topk_slice;
+  c->nsplit_attn = c->tc ? (SM_SLOTS / (f.n_heads * B) < 1 ? 1 : (SM_SLOTS / (f.n_heads * B) > 16 ? 16 : SM_SLOTS / (f.n_heads * B))) : 1;
+  int Mlog = (int)round_up((size_t)B * T, 16);
+  c->keep_logits = !c->tc || (f.flags & SPEC_FLAG_KEEP_LOGITS) || f.accept_mode == 1;
+  size_t M = c->Mcap;
+
+  c->d_status = b.take<int>(4);
+  c->d_n = b.take<int>(B); c->d_cnt = b.take<int>(B); c->d_n_old = b.take<int>(B); c->d_root = b.take<int>(B);
+  c->d_count = b.take<int>(B); c->d_path = b.take<int>((size_t)B * (K + 1)); c->d_out_tok = b.take<int>((size_t)B * (K + 1));
+  c->d_gen_cnt = b.take<int>(B); c->d_gen_log = b.take<int>((size_t)B * c->gen_cap);
+  c->d_cand = b.take<int>((size_t)B * (K + 1) * c->kmax); c->d_cand_ov = b.take<int>((size_t)B * (K ? K : 1) * c->kmax);
+  c->d_tok = b.take<int>(M); c->d_pos = b.take<int>(M); c->d_slot = b.take<int>(M); c->d_am = b.take<int>(M);
+  c->d_edge = b.take<int>(M);
+  c->d_parent = b.take<int>(SPEC_MAX_NODES); c->d_depth = b.take<int>(SPEC_MAX_NODES); c->d_rank = b.take<int>(SPEC_MAX_NODES);
+  c->d_anc_tree = b.take<uint32_t>(SPEC_MAX_NODES * 4); c->d_anc_chain = b.take<uint32_t>(PREFILL_ROWS * 4);
+  c->d_page_table = b.take<int>((size_t)B * c->pages_per_seq);
+  c->d_prompt = b.take<int>((size_t)B * f.max_seq); c->d_offsets = b.take<int>(B + 1);
+  c->d_mw = b.take<const void*>(SPEC_MAX_HEADS); c->d_mb = b.take<const void*>(SPEC_MAX_HEADS);
+  c->d_x = b.take<float>(M * d, 1024); c->d_hid = b.take<float>(M * d, 1024); c->d_h_last = b.take<float>((size_t)B * d);
+  // split-K / plain projection outputs
+  size_t pf = 0;
+  {
+    int Ms[3] = {B * T, B * PREFILL_ROWS, B};
+    for (int i = 0; i < 3; ++i) {
+      size_t m = Ms[i];
+      if (c->tc) {
+        int mt = mt_for_rows((int)m), mtiles = ((int)m + mt - 1) / mt;
+        size_t a = (size_t)splits_for((c->Nqkv + 127) / 128, mtiles, d) * m * c->Nqkv;
+        size_t o = (size_t)splits_for((d + 127) / 128, mtiles, HD) * m * d;
+        size_t dn = (size_t)splits_for((d + 127) / 128, mtiles, F) * m * d;
+        pf = std::max(pf, std::max(a, std::max(o, dn)));
+      } else {
+        pf = std::max(pf, std::max(m * (size_t)c->Nqkv, 2 * m * (size_t)F));
+      }
+    }
+  }
+  c->part_floats = pf;
+  c->d_part = b.take<float>(pf, 1024);
+  c->d_logits = c->keep_logits ? b.take<float>((size_t)Mlog * V, 1024) : nullptr;
+  c->d_pval = b.take<float>((size_t)c->ntile_lm * M); c->d_pidx = b.take<int>((size_t)c->ntile_lm * M);
+  c->d_part_o = c->tc ? b.take<float>((size_t)c->nsplit_attn * M * HD, 1024) : nullptr;
+  c->d_part_ml = c->tc ? b.take<float>((size_t)c->nsplit_attn * M * f.n_heads * 2) : nullptr;
+  c->d_pk_val = b.take<float>((size_t)c->topk_blocks * B * (K ? K : 1) * c->kmax);
+  c->d_pk_idx = b.take<int>((size_t)c->topk_blocks * B * (K ? K : 1) * c->kmax);
+  c->d_rope = b.take<float2>((size_t)c->cap * (f.head_dim / 2));
+  size_t e = c->esz;
+  c->d_u = b.take<uint8_t>(M * d * e, 1024); c->d_q = b.take<uint8_t>(M * HD * e, 1024);
+  c->d_attn = b.take<uint8_t>(M * HD * e, 1024); c->d_act = b.take<uint8_t>(M * F * e, 1024);
+  c->d_hq = b.take<uint8_t>(M * d * e, 1024); c->d_hq_last = b.take<uint8_t>(round_up((size_t)B, 16) * d * e, 1024);
+  c->d_r = b.take<uint8_t>((size_t)B * (K ? K : 1) * d * e, 1024);
+  c->geom = KVGeom{f.n_layers, f.n_kv_heads, f.head_dim, f.page_size, c->pages_per_seq, B};
+  size_t pool_elems = (size_t)B * c->pages_per_seq * c->geom.page_elems();
+  c->d_pool = b.take<uint8_t>(pool_elems * e, 1024);
+  return round_up(b.off, 1024);
+}
+
+#define CUDA_OK(call)                                                                          \
+  do {                                                                                         \
+    cudaError_t e_ = (call);                                                                   \
+    if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); \
+  } while (0)
+
+#define LAUNCH_CHECK(name)                                                                     \
+  do {                                                                                         \
+    c->launches++;                                                                             \
+    cudaError_t e_ = cudaGetLastError();                                                       \
+    if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string(name) + ": " + cudaGetErrorString(e_)); \
+  } while (0)
+
+Rows make_rows(spec_ctx* c, int R, bool chain) {
+  Rows r;
+  r.R = R; r.B = c->B;
+  r.tok = c->d_tok; r.pos = c->d_pos; r.slot = c->d_slot; r.n = c->d_n; r.cnt = c->d_cnt;
+  r.anc = chain ? c->d_anc_chain : c->d_anc_tree;
+  return r;
+}
+
+// ---- tensor-core linear launch (bf16) ----
+template <int MT, int EPI>
+int launch_gemm_tc_mt(spec_ctx* c, cudaStream_t st, const CUtensorMap* a, const CUtensorMap* a2, const CUtensorMap* bm,
+                      const GemmTcParams& p, int n_tiles, int m_tiles, long long* launches) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc<MT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmTcCfg<MT>::SMEM_BYTES) != cudaSuccess)
+      return SPEC_E_CUDA;
+    attr_set = true;
+  }
+  dim3 grid(n_tiles, p.splits, m_tiles);
+  gemm_tc<MT, EPI><<<grid, 128, GemmTcCfg<MT>::SMEM_BYTES, st>>>(*a, *a2, *bm, p);
+  if (launches) ++*launches;
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_E_CUDA;
+}
+template <int EPI>
+int launch_gemm_tc(spec_ctx* c, cudaStream_t st, int mt, const CUtensorMap* a, const CUtensorMap* a2, const CUtensorMap* bm,
+                   const GemmTcParams& p, int n_tiles, int m_tiles, long long* launches) {
+  switch (mt) {
+    case 16: return launch_gemm_tc_mt<16, EPI>(c, st, a, a2, bm, p, n_tiles, m_tiles, launches);
+    case 32: return launch_gemm_tc_mt<32, EPI>(c, st, a, a2, bm, p, n_tiles, m_tiles, launches);
+    case 64: return launch_gemm_tc_mt<64, EPI>(c, st, a, a2, bm, p, n_tiles, m_tiles, launches);
+    default: return launch_gemm_tc_mt<128, EPI>(c, st, a, a2, bm, p, n_tiles, m_tiles, launches);
+  }
+}
+
+// y partials = x[M,K] W[N,K]^T; returns the number of K slices used (>0) or a negative error.
+int linear_tc_partial(spec_ctx* c, const void* x, const void* W, int M, int N, int K, float* out) {
+  int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (N + 127) / 128;
+  int s = splits_for(n_tiles, m_tiles, K);
+  if ((size_t)s * M * N > c->part_floats && out == c->d_part) return c->fail(SPEC_E_NOMEM, "split-K scratch too small");
+  const CUtensorMap* ta = c->tmap(W, N, K, 64);
+  const CUtensorMap* tb = c->tmap(x, std::max<size_t>(round_up(M, 16), mt), K, mt);
+  if (!ta || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
+  GemmTcParams p{};
+  p.M = M; p.N = N; p.K = K; p.splits = s; p.a2_row_offset = 64; p.tile_rows = 128;
+  p.out = out; p.split_stride = (size_t)M * N; p.ldo = N; p.status = c->d_status;
+  if (launch_gemm_tc<EPI_PARTIAL>(c, c->stream, mt, ta, ta, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
+    return c->fail(SPEC_E_CUDA, std::string("gemm_tc launch: ") + cudaGetErrorString(cudaGetLastError()));
+  return s;
+}
+
+template <typename T>
+int linear_simple(spec_ctx* c, const T* x, int ldx, const T* W, float* y, int ldy, int M, int N, int K) {
+  constexpr int MC = 8;
+  dim3 grid((N + 7) / 8, (M + MC - 1) / MC);
+  linear_rows<T, MC><<<grid, 256, 0, c->stream>>>(x, ldx, W, y, ldy, M, N, K);
+  LAUNCH_CHECK("linear_rows");
+  return SPEC_OK;
+}
+
+// One pass of the base model over M = B*R rows whose tokens/positions/slots are prepared
+// and whose embeddings are in d_x. lm_rows > 0: run lm_head over the first lm_rows rows of
+// `lm_src` (bf16/float operand rows) and leave per-row argmax partials.
+template <typename T>
+int forward_layers(spec_ctx* c, int R, bool chain) {
+  const spec_config& f = c->cfg;
+  Rows rows = make_rows(c, R, chain);
+  int M = c->B * R, d = f.d_model, F = f.d_ffn, H = f.n_heads, D = f.head_dim, HD = H * D;
+  T* u = static_cast<T*>(c->d_u);
+  T* q = static_cast<T*>(c->d_q);
+  T* attn = static_cast<T*>(c->d_attn);
+  T* act = static_cast<T*>(c->d_act);
+  T* pool = static_cast<T*>(c->d_pool);
+  int pending = 0;              // K slices of the previous down-projection still to be added to x
+  size_t pending_stride = 0;
+  for (int l = 0; l < f.n_layers; ++l) {
+    rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, pending, pending_stride, c->an[l], f.rms_eps, u, nullptr, d);
+    LAUNCH_CHECK("rmsnorm_rows");
+    int sq = 1;
+    if (c->tc) {
+      if (c->qkv_fused) {
+        sq = linear_tc_partial(c, u, c->wq[l], M, c->Nqkv, d, c->d_part);
+        if (sq < 0) return sq;
+      } else {
+        return c->fail(SPEC_E_BADARG, "bf16 path needs wq/wk/wv contiguous per layer");
+      }
+    } else {
+      int nk = f.n_kv_heads * D, r;
+      if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wq[l]), c->d_part, c->Nqkv, M, HD, d))) return r;
+      if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wk[l]), c->d_part + HD, c->Nqkv, M, nk, d))) return r;
+      if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wv[l]), c->d_part + HD + nk, c->Nqkv, M, nk, d))) return r;
+    }
+    rope_store<T><<<M, 256, 0, c->stream>>>(c->d_part, sq, (size_t)M * c->Nqkv, rows, c->d_rope, q, pool, c->geom, c->d_page_table, l, H);
+    LAUNCH_CHECK("rope_store");
+    if (c->tc) {
+      AttnTcArgs a{};
+      a.q = reinterpret_cast<const bf16*>(q); a.part_o = c->d_part_o; a.part_ml = c->d_part_ml;
+      a.pool = reinterpret_cast<const bf16*>(pool); a.g = c->geom; a.page_table = c->d_page_table; a.rows = rows;
+      a.layer = l; a.H = H; a.nsplit = c->nsplit_attn; a.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+      a.status = c->d_status;
+      dim3 grid(H, c->nsplit_attn, c->B);
+      int nw = (R + 15) / 16;
+      size_t rowb = (size_t)D * 2;
+#define ATTN_CASE(HDV, NWV)                                                                              \
+      {                                                                                                  \
+        size_t sm = (size_t)NWV * 16 * rowb + 4 * 64 * rowb + 64;                                        \
+        static bool set_ = false;                                                                        \
+        if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_tc<HDV, NWV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); set_ = true; } \
+        attention_tc<HDV, NWV><<<grid, NWV * 32, sm, c->stream>>>(a);                                    \
+      }
+      if (D == 128) {
+        if (nw <= 1) ATTN_CASE(128, 1) else if (nw <= 2) ATTN_CASE(128, 2) else if (nw <= 4) ATTN_CASE(128, 4) else ATTN_CASE(128, 8)
+      } else {
+        if (nw <= 1) ATTN_CASE(64, 1) else if (nw <= 2) ATTN_CASE(64, 2) else if (nw <= 4) ATTN_CASE(64, 4) else ATTN_CASE(64, 8)
+      }
+#undef ATTN_CASE
+      LAUNCH_CHECK("attention_tc");
+      size_t total = (size_t)M * HD / 4;
+      attention_combine<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(c->d_part_o, c->d_part_ml, c->nsplit_attn, rows, H, D,
+                                                                                reinterpret_cast<bf16*>(attn));
+      LAUNCH_CHECK("attention_combine");
+    } else {
+      dim3 grid(H, c->B, (R + 3) / 4);
+      attention_simple<T><<<grid, 128, 0, c->stream>>>(q, attn, pool, c->geom, c->d_page_table, rows, l, H, 1.0f / sqrtf((float)D));
+      LAUNCH_CHECK("attention_simple");
+    }
+    // output projection + residual + FFN norm
+    int so = 1;
+    if (c->tc) { so = linear_tc_partial(c, attn, c->wo[l], M, d, HD, c->d_part); if (so < 0) return so; }
+    else { int r = linear_simple<T>(c, attn, HD, static_cast<const T*>(c->wo[l]), c->d_part, d, M, d, HD); if (r) return r; }
+    rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, so, (size_t)M * d, c->fn[l], f.rms_eps, u, nullptr, d);
+    LAUNCH_CHECK("rmsnorm_rows");
+    // SwiGLU FFN
+    if (c->tc) {
+      int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (F + 63) / 64;
+      const CUtensorMap* tg = c->tmap(c->wg[l], F, d, 64);
+      const CUtensorMap* tu = c->tmap(c->wu[l], F, d, 64);
+      const CUtensorMap* tb = c->tmap(u, std::max<size_t>(round_up(M, 16), mt), d, mt);
+      if (!tg || !tu || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
+      GemmTcParams p{};
+      p.M = M; p.N = F; p.K = d; p.splits = 1; p.a2_row_offset = 0; p.tile_rows = 64;
+      p.act = reinterpret_cast<bf16*>(act); p.ld_act = F; p.status = c->d_status;
+      if (launch_gemm_tc<EPI_SWIGLU>(c, c->stream, mt, tg, tu, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
+        return c->fail(SPEC_E_CUDA, std::string("gemm_tc swiglu launch: ") + cudaGetErrorString(cudaGetLastError()));
+    } else {
+      float* g = c->d_part;
+      float* up = c->d_part + (size_t)M * F;
+      int r;
+      if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wg[l]), g, F, M, F, d))) return r;
+      if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wu[l]), up, F, M, F, d))) return r;
+      size_t total = (size_t)M * F;
+      swiglu_rows<T><<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(g, up, act, total);
+      LAUNCH_CHECK("swiglu_rows");
+    }
+    if (c->tc) { pending = linear_tc_partial(c, act, c->wd[l], M, d, F, c->d_part); if (pending < 0) return pending; }
+    else { int r = linear_simple<T>(c, act, F, static_cast<const T*>(c->wd[l]), c->d_part, d, M, d, F); if (r) return r; pending = 1; }
+    pending_stride = (size_t)M * d;
+  }
+  // final norm: hidden (float32) and its operand-typed copy
+  rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, pending, pending_stride, c->final_norm, f.rms_eps,
+                                            static_cast<T*>(c->d_hq), c->d_hid, d);
+  LAUNCH_CHECK("rmsnorm_rows");
+  return SPEC_OK;
+}
+
+// lm_head over `M` operand rows at `src`, leaving per-row argmax partials (and logits).
+template <typename T>
+int lm_head_argmax(spec_ctx* c, const T* src, int M) {
+  const spec_config& f = c->cfg;
+  if (c->tc) {
+    int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = c->ntile_lm;
+    const CUtensorMap* ta = c->tmap(c->lm_head, f.vocab, f.d_model, 64);
+    const CUtensorMap* tb = c->tmap(src, std::max<size_t>(round_up(M, 16), mt), f.d_model, mt);
+    if (!ta || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
+    GemmTcParams p{};
+    p.M = M; p.N = f.vocab; p.K = f.d_model; p.splits = 1; p.a2_row_offset = 64; p.tile_rows = 128;
+    p.logits = c->keep_logits ? c->d_logits : nullptr; p.pval = c->d_pval; p.pidx = c->d_pidx; p.pstride = c->Mcap;
+    p.status = c->d_status;
+    if (launch_gemm_tc<EPI_ARGMAX>(c, c->stream, mt, ta, ta, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
+      return c->fail(SPEC_E_CUDA, std::string("gemm_tc lm_head launch: ") + cudaGetErrorString(cudaGetLastError()));
+  } else {
+    int r = linear_simple<T>(c, src, f.d_model, static_cast<const T*>(c->lm_head), c->d_logits, f.vocab, M, f.vocab, f.d_model);
+    if (r) return r;
+    argmax_rows<<<M, 256, 0, c->stream>>>(c->d_logits, f.vocab, c->d_pval, c->d_pidx);
+    LAUNCH_CHECK("argmax_rows");
+  }
+  return SPEC_OK;
+}
+
+AcceptArgs make_accept(spec_ctx* c, int R, int mode) {
+  AcceptArgs a{};
+  a.rows = make_rows(c, R, false);
+  a.pval = c->d_pval; a.pidx = c->d_pidx; a.ntile = c->ntile_lm; a.pstride = c->Mcap;
+  a.parent = c->d_parent; a.depth = c->d_depth; a.edge_ok = nullptr;
+  a.K = c->K; a.frag_token = c->cfg.frag_token; a.d = c->cfg.d_model; a.mode = mode;
+  a.hid = c->d_hid; a.am = c->d_am; a.path = c->d_path; a.count = c->d_count; a.out_tok = c->d_out_tok;
+  a.n_old = c->d_n_old; a.root_tok = c->d_root; a.h_last = c->d_h_last;
+  a.gen_log = c->d_gen_log; a.gen_cnt = c->d_gen_cnt; a.gen_cap = c->gen_cap;
+  return a;
+}
+
+int check_status(spec_ctx* c) {
+  int st[4];
+  cudaError_t e = cudaMemcpyAsync(st, c->d_status, sizeof(st), cudaMemcpyDeviceToHost, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("status read: ") + cudaGetErrorString(e));
+  if (st[0] == ST_OK) return SPEC_OK;
+  char buf[128];
+  snprintf(buf, sizeof(buf), "device status %d at %d (detail %d)", st[0], st[1], st[2]);
+  return c->fail(st[0] == ST_TIMEOUT ? SPEC_E_TIMEOUT : (st[0] == ST_SEQLEN ? SPEC_E_SEQLEN : SPEC_E_BADARG), buf);
+}
+
+template <typename T>
+int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offsets) {
+  const spec_config& f = c->cfg;
+  int maxlen = 0;
+  for (int b = 0; b < batch; ++b) {
+    int len = offsets[b + 1] - offsets[b];
+    if (len < 1) return c->fail(SPEC_E_BADARG, "empty prompt");
+    if (len + c->K + 1 > f.max_seq) return c->fail(SPEC_E_SEQLEN, "prompt leaves no room to generate within max_seq");
+    if (offsets[b + 1] - offsets[0] > batch * f.max_seq) return c->fail(SPEC_E_SEQLEN, "prompts exceed the prompt buffer");
+    maxlen = std::max(maxlen, len);
+  }
+  c->B = batch;
+  c->prefilled = false;
+  std::vector<int> off(batch + 1);
+  for (int b = 0; b <= batch; ++b) off[b] = offsets[b] - offsets[0];
+  CUDA_OK(cudaMemsetAsync(c->d_status, 0, 4 * sizeof(int), c->stream));
+  CUDA_OK(cudaMemsetAsync(c->d_pool, 0, (size_t)f.max_batch * c->pages_per_seq * c->geom.page_elems() * c->esz, c->stream));
+  CUDA_OK(cudaMemcpyAsync(c->d_prompt, tokens + offsets[0], (size_t)off[batch] * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_OK(cudaMemcpyAsync(c->d_offsets, off.data(), (batch + 1) * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_OK(cudaMemsetAsync(c->d_gen_cnt, 0, batch * sizeof(int), c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));   // host staging vector goes out of scope below
+  int R = PREFILL_ROWS, M = batch * R;
+  Rows rows = make_rows(c, R, true);
+  int chunks = (maxlen + R - 1) / R;
+  for (int ch = 0; ch < chunks; ++ch) {
+    prepare_prefill_rows<T><<<M, 128, 0, c->stream>>>(rows, c->d_prompt, c->d_offsets, ch, static_cast<const T*>(c->embed), c->d_x,
+                                                    f.d_model, f.vocab, c->d_status);
+    LAUNCH_CHECK("prepare_prefill_rows");
+    int r = forward_layers<T>(c, R, true);
+    if (r) return r;
+    prefill_keep_last<T><<<batch, 256, 0, c->stream>>>(rows, c->d_offsets, ch, c->d_hid, c->d_h_last, static_cast<T*>(c->d_hq_last), f.d_model);
+    LAUNCH_CHECK("prefill_keep_last");
+  }
+  int r = lm_head_argmax<T>(c, static_cast<const T*>(c->d_hq_last), batch);
+  if (r) return r;
+  AcceptArgs a = make_accept(c, 1, 1);
+  accept_kernel<<<batch, 128, 0, c->stream>>>(a);
+  LAUNCH_CHECK("accept_kernel");
+  r = check_status(c);
+  if (r) return r;
+  c->n_hi.assign(batch, 0);
+  for (int b = 0; b < batch; ++b) c->n_hi[b] = offsets[b + 1] - offsets[b];
+  c->prefilled = true;
+  return SPEC_OK;
+}
+
+template <typename T>
+int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t* cand_override) {
+  const spec_config& f = c->cfg;
+  int B = c->B, K = c->K, T_ = c->T, d = f.d_model, kmax = c->kmax;
+  for (int b = 0; b < B; ++b)
+    if (c->n_hi[b] + K + 1 > f.max_seq) return c->fail(SPEC_E_SEQLEN, "sequence would exceed max_seq");
+  const int* ov = nullptr;
+  if (cand_override && K > 0) {
+    CUDA_OK(cudaMemcpyAsync(c->d_cand_ov, cand_override, (size_t)B * K * kmax * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    ov = c->d_cand_ov;
+  }
+  // (1) extra heads -> shared lm_head -> per-head top-k -> candidate table
+  if (K > 0) {
+    constexpr int MC = 4;
+    dim3 g1((K * d + 7) / 8, (B + MC - 1) / MC);
+    medusa_resblock<T, MC><<<g1, 256, 0, c->stream>>>(c->d_h_last, reinterpret_cast<const T* const*>(c->d_mw),
+                                                    reinterpret_cast<const T* const*>(c->d_mb), static_cast<T*>(c->d_r), B, K, d);
+    LAUNCH_CHECK("medusa_resblock");
+    int rows_total = B * K;
+    dim3 g2(c->topk_blocks, (rows_total + MC - 1) / MC);
+    size_t sm = (size_t)MC * c->topk_slice * sizeof(float);
+    medusa_lmhead_topk<T, MC><<<g2, 256, sm, c->stream>>>(static_cast<const T*>(c->d_r), static_cast<const T*>(c->lm_head), rows_total,
+                                                        f.vocab, d, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
+    LAUNCH_CHECK("medusa_lmhead_topk");
+    // partial lists of the row chunks are laid out per block over all rows
+    size_t sm2 = (size_t)c->topk_blocks * kmax * 8;
+    topk_merge<<<rows_total, 256, sm2, c->stream>>>(c->d_pk_val, c->d_pk_idx, c->topk_blocks, rows_total, K, kmax, c->d_root, ov, c->d_cand);
+    LAUNCH_CHECK("topk_merge");
+  } else {
+    CUDA_OK(cudaMemcpyAsync(c->d_cand, c->d_root, B * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  }
+  // (2) candidate tree -> rows
+  int M = B * T_;
+  Rows rows = make_rows(c, T_, false);
+  prepare_verify_rows<T><<<M, 128, 0, c->stream>>>(rows, c->d_cand, (K + 1) * kmax, kmax, c->d_depth, c->d_rank, c->cap,
+                                                 static_cast<const T*>(c->embed), c->d_x, d, f.vocab, c->d_status);
+  LAUNCH_CHECK("prepare_verify_rows");
+  // (3) verification forward
+  int r = forward_layers<T>(c, T_, false);
+  if (r) return r;
+  r = lm_head_argmax<T>(c, static_cast<const T*>(c->d_hq), M);
+  if (r) return r;
+  // (4) acceptance
+  AcceptArgs a = make_accept(c, T_, 0);
+  if (f.accept_mode == 1) {
+    typical_edges<<<M, 256, 0, c->stream>>>(c->d_logits, f.vocab, rows, c->d_parent, f.typ_eps, f.typ_delta,
+                                            1.0f / (f.temperature > 0.f ? f.temperature : 1.0f), c->d_edge);
+    LAUNCH_CHECK("typical_edges");
+    a.edge_ok = c->d_edge;
+  }
+  accept_kernel<<<B, 128, 0, c->stream>>>(a);
+  LAUNCH_CHECK("accept_kernel");
+  // (5) KV compaction
+  dim3 gc(f.n_layers * 2 * f.n_kv_heads, B);
+  compact_kv<T><<<gc, 64, 0, c->stream>>>(static_cast<T*>(c->d_pool), c->geom, c->d_page_table, c->d_path, c->d_count, c->d_n_old, K);
+  LAUNCH_CHECK("compact_kv");
+  if (out_tokens || out_counts) {
+    if (out_tokens) CUDA_OK(cudaMemcpyAsync(out_tokens, c->d_out_tok, (size_t)B * (K + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    if (out_counts) CUDA_OK(cudaMemcpyAsync(out_counts, c->d_count, (size_t)B * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    std::vector<int> nn(B);
+    CUDA_OK(cudaMemcpyAsync(nn.data(), c->d_n, B * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    r = check_status(c);   // synchronises
+    if (r) return r;
+    for (int b = 0; b < B; ++b) c->n_hi[b] = nn[b];
+  } else {
+    for (int b = 0; b < B; ++b) c->n_hi[b] += K + 1;
+  }
+  return SPEC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t spec_workspace_bytes(const spec_config* cfg, const spec_tree* tree) {
+  std::string why;
+  if (!cfg || !tree || !validate_config(cfg, &why)) return 0;
+  spec_ctx tmp{};
+  tmp.cfg = *cfg;
+  if (!validate_tree(cfg, tree, &tmp.kmax, &why)) return 0;
+  tmp.T = tree->n_nodes; tmp.K = cfg->n_medusa;
+  tmp.tc = cfg->dtype == 1 && !(cfg->flags & SPEC_FLAG_SIMPLE_KERNELS);
+  tmp.esz = cfg->dtype == 1 ? 2 : 4;
+  return carve(&tmp, nullptr);
+}
+
+int spec_create(const spec_config* cfg, const spec_weights* w, const spec_tree* tree, void* workspace,
+                size_t workspace_bytes, void* cuda_stream, spec_ctx** out) {
+  std::string why;
+  if (!cfg || !w || !tree || !workspace || !out) { g_create_error = "null argument"; return SPEC_E_BADARG; }
+  if (!validate_config(cfg, &why)) { g_create_error = why; return SPEC_E_BADARG; }
+  int kmax = 1;
+  if (!validate_tree(cfg, tree, &kmax, &why)) { g_create_error = why; return SPEC_E_BADTREE; }
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo ||
+      !w->ffn_norm || !w->w_gate || !w->w_up || !w->w_down || (cfg->n_medusa > 0 && (!w->medusa_w || !w->medusa_b))) {
+    g_create_error = "null weight pointer"; return SPEC_E_BADARG;
+  }
+  if (reinterpret_cast<uintptr_t>(workspace) % 1024) { g_create_error = "workspace must be 1024-byte aligned"; return SPEC_E_BADARG; }
+  spec_ctx* c = new spec_ctx();
+  c->cfg = *cfg;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->T = tree->n_nodes; c->K = cfg->n_medusa; c->kmax = kmax; c->B = cfg->max_batch;
+  c->tc = cfg->dtype == 1 && !(cfg->flags & SPEC_FLAG_SIMPLE_KERNELS);
+  c->esz = cfg->dtype == 1 ? 2 : 4;
+  size_t need = carve(c, workspace);
+  if (need > workspace_bytes) { g_create_error = "workspace too small"; delete c; return SPEC_E_NOMEM; }
+  c->h_parent.assign(tree->parent, tree->parent + c->T);
+  c->h_depth.assign(tree->depth, tree->depth + c->T);
+  c->h_rank.assign(tree->rank, tree->rank + c->T);
+  int L = cfg->n_layers;
+  c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
+  c->qkv_fused = true;
+  size_t qn = (size_t)cfg->n_heads * cfg->head_dim * cfg->d_model * c->esz, kn = (size_t)cfg->n_kv_heads * cfg->head_dim * cfg->d_model * c->esz;
+  for (int l = 0; l < L; ++l) {
+    if (!w->attn_norm[l] || !w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->ffn_norm[l] || !w->w_gate[l] || !w->w_up[l] || !w->w_down[l]) {
+      g_create_error = "null layer weight pointer"; delete c; return SPEC_E_BADARG;
+    }
+    c->an.push_back(w->attn_norm[l]); c->fn.push_back(w->ffn_norm[l]);
+    c->wq.push_back(w->wq[l]); c->wk.push_back(w->wk[l]); c->wv.push_back(w->wv[l]); c->wo.push_back(w->wo[l]);
+    c->wg.push_back(w->w_gate[l]); c->wu.push_back(w->w_up[l]); c->wd.push_back(w->w_down[l]);
+    const uint8_t* q0 = static_cast<const uint8_t*>(w->wq[l]);
+    if (static_cast<const uint8_t*>(w->wk[l]) != q0 + qn || static_cast<const uint8_t*>(w->wv[l]) != q0 + qn + kn) c->qkv_fused = false;
+  }
+  for (int k = 0; k < c->K; ++k) { c->mw.push_back(w->medusa_w[k]); c->mb.push_back(w->medusa_b[k]); }
+  if (c->tc && !c->qkv_fused) { g_create_error = "bf16 path needs wq/wk/wv of a layer contiguous (wq, wk, wv)"; delete c; return SPEC_E_BADARG; }
+  if (c->tc && !get_encode_fn()) { g_create_error = "cuTensorMapEncodeTiled entry point unavailable"; delete c; return SPEC_E_CUDA; }
+
+  // host-made tables: tree arrays, ancestor bitsets (tree and chain), page table, RoPE table
+  std::vector<uint32_t> anc_tree(SPEC_MAX_NODES * 4, 0), anc_chain(PREFILL_ROWS * 4, 0);
+  for (int v = 0; v < c->T; ++v) {
+    if (v > 0) for (int wd = 0; wd < 4; ++wd) anc_tree[v * 4 + wd] = anc_tree[c->h_parent[v] * 4 + wd];
+    anc_tree[v * 4 + (v >> 5)] |= 1u << (v & 31);
+  }
+  for (int v = 0; v < PREFILL_ROWS; ++v)
+    for (int u = 0; u <= v; ++u) anc_chain[v * 4 + (u >> 5)] |= 1u << (u & 31);
+  std::vector<int> pt((size_t)cfg->max_batch * c->pages_per_seq);
+  for (int b = 0; b < cfg->max_batch; ++b)
+    for (int p = 0; p < c->pages_per_seq; ++p) pt[(size_t)b * c->pages_per_seq + p] = p * cfg->max_batch + b;
+  int half = cfg->head_dim / 2;
+  std::vector<float2> rope((size_t)c->cap * half);
+  for (int i = 0; i < half; ++i) {
+    double inv = pow((double)cfg->rope_base, -2.0 * i / cfg->head_dim);
+    for (int p = 0; p < c->cap; ++p) {
+      double ang = (double)p * inv;
+      rope[(size_t)p * half + i] = make_float2((float)cos(ang), (float)sin(ang));
+    }
+  }
+  cudaError_t e = cudaSuccess;
+  auto up = [&](void* dst, const void* src, size_t bytes) {
+    if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, c->stream);
+  };
+  up(c->d_parent, c->h_parent.data(), c->T * sizeof(int));
+  up(c->d_depth, c->h_depth.data(), c->T * sizeof(int));
+  up(c->d_rank, c->h_rank.data(), c->T * sizeof(int));
+  up(c->d_anc_tree, anc_tree.data(), anc_tree.size() * 4);
+  up(c->d_anc_chain, anc_chain.data(), anc_chain.size() * 4);
+  up(c->d_page_table, pt.data(), pt.size() * sizeof(int));
+  up(c->d_rope, rope.data(), rope.size() * sizeof(float2));
+  up(c->d_mw, c->mw.data(), c->mw.size() * sizeof(void*));
+  up(c->d_mb, c->mb.data(), c->mb.size() * sizeof(void*));
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 4 * sizeof(int), c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_cand, 0, (size_t)cfg->max_batch * (c->K + 1) * c->kmax * sizeof(int), c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) { g_create_error = std::string("set-up copies: ") + cudaGetErrorString(e); delete c; return SPEC_E_CUDA; }
+  *out = c;
+  return SPEC_OK;
+}
+
+int spec_prefill(spec_ctx* c, int32_t batch, const int32_t* tokens, const int32_t* offsets) {
+  if (!c) return SPEC_E_BADARG;
+  if (!tokens || !offsets) return c->fail(SPEC_E_BADARG, "null argument");
+  if (batch < 1 || batch > c->cfg.max_batch) return c->fail(SPEC_E_BADARG, "batch out of range");
+  return c->cfg.dtype == 1 ? prefill_t<bf16>(c, batch, tokens, offsets) : prefill_t<float>(c, batch, tokens, offsets);
+}
+
+int spec_step(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t* cand_override) {
+  if (!c) return SPEC_E_BADARG;
+  if (!c->prefilled) return c->fail(SPEC_E_STATE, "spec_step before spec_prefill");
+  return c->cfg.dtype == 1 ? step_t<bf16>(c, out_tokens, out_counts, cand_override)
+                           : step_t<float>(c, out_tokens, out_counts, cand_override);
+}
+
+int spec_read_generated(spec_ctx* c, int32_t seq, int32_t* out, int32_t max_tokens, int32_t* n_generated) {
+  if (!c) return SPEC_E_BADARG;
+  if (!c->prefilled) return c->fail(SPEC_E_STATE, "nothing generated yet");
+  if (seq < 0 || seq >= c->B || !n_generated || max_tokens < 0) return c->fail(SPEC_E_BADARG, "bad argument");
+  int r = check_status(c);
+  if (r) return r;
+  int cnt = 0;
+  CUDA_OK(cudaMemcpyAsync(&cnt, c->d_gen_cnt + seq, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  int stored = cnt < c->gen_cap ? cnt : c->gen_cap;
+  int ncopy = stored < max_tokens ? stored : max_tokens;
+  if (out && ncopy > 0) {
+    CUDA_OK(cudaMemcpyAsync(out, c->d_gen_log + (size_t)seq * c->gen_cap, ncopy * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_OK(cudaStreamSynchronize(c->stream));
+  }
+  *n_generated = cnt;
+  std::vector<int> nn(c->B);
+  CUDA_OK(cudaMemcpyAsync(nn.data(), c->d_n, c->B * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  for (int b = 0; b < c->B; ++b) c->n_hi[b] = nn[b];
+  return SPEC_OK;
+}
+
+int spec_destroy(spec_ctx* c) {
+  if (!c) return SPEC_E_BADARG;
+  cudaStreamSynchronize(c->stream);
+  delete c;
+  return SPEC_OK;
+}
+
+const char* spec_last_error(const spec_ctx* c) { return c ? c->err.c_str() : g_create_error.c_str(); }
+
+int64_t spec_query(const spec_ctx* c, int32_t what) {
+  if (!c) return -1;
+  const spec_config& f = c->cfg;
+  switch (what) {
+    case SPEC_Q_KMAX: return c->kmax;
+    case SPEC_Q_KERNEL_LAUNCHES: return c->launches;
+    case SPEC_Q_N_NODES: return c->T;
+    case SPEC_Q_BATCH: return c->B;
+    case SPEC_Q_ALGO_BYTES_PER_STEP: {
+      double d = f.d_model, F = f.d_ffn, V = f.vocab, HD = (double)f.n_heads * f.head_dim, KD = (double)f.n_kv_heads * f.head_dim;
+      double layer = d * HD + 2 * d * KD + HD * d + 3 * d * F;
+      double bytes = (f.n_layers * layer + 2 * V * d + c->K * (d * d + d)) * (double)c->esz;
+      return (int64_t)(bytes / 1024.0);
+    }
+    default: return -1;
+  }
+}
+
+int spec_debug_read(spec_ctx* c, int32_t what, void* host_buf, size_t bytes) {
+  if (!c || !host_buf) return SPEC_E_BADARG;
+  const spec_config& f = c->cfg;
+  size_t rows = (size_t)c->B * c->T;
+  const void* src = nullptr;
+  size_t need = 0;
+  switch (what) {
+    case SPEC_DBG_TOK: src = c->d_tok; need = rows * 4; break;
+    case SPEC_DBG_POS: src = c->d_pos; need = rows * 4; break;
+    case SPEC_DBG_LOGITS: src = c->d_logits; need = rows * f.vocab * 4; break;
+    case SPEC_DBG_HIDDEN: src = c->d_hid; need = rows * f.d_model * 4; break;
+    case SPEC_DBG_ARGMAX: src = c->d_am; need = rows * 4; break;
+    case SPEC_DBG_PATH: src = c->d_path; need = (size_t)c->B * (c->K + 1) * 4; break;
+    case SPEC_DBG_CAND: src = c->d_cand; need = (size_t)c->B * (c->K + 1) * c->kmax * 4; break;
+    case SPEC_DBG_SEQLEN: src = c->d_n; need = (size_t)c->B * 4; break;
+    case SPEC_DBG_NEXT_ROOT: src = c->d_root; need = (size_t)c->B * 4; break;
+    case SPEC_DBG_H_LAST: src = c->d_h_last; need = (size_t)c->B * f.d_model * 4; break;
+    case SPEC_DBG_STATUS: src = c->d_status; need = 16; break;
+    default: return c->fail(SPEC_E_BADARG, "unknown debug tap");
+  }
+  if (!src) return c->fail(SPEC_E_STATE, "tap not available (logits need SPEC_FLAG_KEEP_LOGITS)");
+  if (bytes < need) return c->fail(SPEC_E_BADARG, "host buffer too small");
+  CUDA_OK(cudaMemcpyAsync(host_buf, src, need, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  return SPEC_OK;
+}
+
+int spec_debug_read_kv(spec_ctx* c, int32_t seq, int32_t layer, int32_t slot0, int32_t n_slots, float* host_k, float* host_v) {
+  if (!c || !host_k || !host_v) return SPEC_E_BADARG;
+  const spec_config& f = c->cfg;
+  if (seq < 0 || seq >= f.max_batch || layer < 0 || layer >= f.n_layers || slot0 < 0 || n_slots < 0 || slot0 + n_slots > c->cap)
+    return c->fail(SPEC_E_BADARG, "bad KV range");
+  int D = f.head_dim, Hkv = f.n_kv_heads, ps = f.page_size;
+  std::vector<uint8_t> blk(c->geom.block_elems() * c->esz);
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  for (int kv = 0; kv < 2; ++kv) {
+    float* dst = kv ? host_v : host_k;
+    for (int h = 0; h < Hkv; ++h) {
+      int cur_page = -1;
+      for (int sl = slot0; sl < slot0 + n_slots; ++sl) {
+        int page = (sl / ps) * f.max_batch + seq;   // same mapping as the device page table
+        if (page != cur_page) {
+          const uint8_t* src = static_cast<const uint8_t*>(c->d_pool) + c->geom.block_offset(page, layer, kv, h) * c->esz;
+          CUDA_OK(cudaMemcpy(blk.data(), src, blk.size(), cudaMemcpyDeviceToHost));
+          cur_page = page;
+        }
+        int row = sl % ps;
+        for (int e = 0; e < D; ++e) {
+          float v;
+          if (c->esz == 2) {
+            uint16_t raw = reinterpret_cast<uint16_t*>(blk.data())[(size_t)row * D + kv_elem<bf16>(row, e)];
+            uint32_t u32 = (uint32_t)raw << 16;
+            memcpy(&v, &u32, 4);
+          } else {
+            v = reinterpret_cast<float*>(blk.data())[(size_t)row * D + e];
+          }
+          dst[((size_t)(sl - slot0) * Hkv + h) * D + e] = v;
+        }
+      }
+    }
+  }
+  return SPEC_OK;
+}
+
+int spec_op_linear(int32_t dtype, const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                   int32_t splits, float* scratch, void* cuda_stream) {
+  if (!x || !w || !y || M < 1 || N < 1 || K < 8 || K % 8 || M > 2048) return SPEC_E_BADARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (dtype == 0) {
+    constexpr int MC = 8;
+    dim3 grid((N + 7) / 8, (M + MC - 1) / MC);
+    linear_rows<float, MC><<<grid, 256, 0, st>>>(static_cast<const float*>(x), K, static_cast<const float*>(w), y, N, M, N, K);
+    return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_E_CUDA;
+  }
+  if (dtype != 1 || K % 64 || splits < 1 || splits > K / 64 || !scratch) return SPEC_E_BADARG;
+  if (M % 16) return SPEC_E_BADARG;   // the activation map is declared over whole 16-row groups
+  int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (N + 127) / 128;
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, w, N, K, 64) || !make_tmap(&tb, x, M, K, mt)) return SPEC_E_CUDA;
+  GemmTcParams p{};
+  p.M = M; p.N = N; p.K = K; p.splits = splits; p.a2_row_offset = 64; p.tile_rows = 128;
+  p.out = scratch; p.split_stride = (size_t)M * N; p.ldo = N;
+  // the status word of a stand-alone call lives at the end of the scratch buffer
+  p.status = reinterpret_cast<int*>(scratch + (size_t)splits * M * N);
+  if (cudaMemsetAsync(p.status, 0, 16, st) != cudaSuccess) return SPEC_E_CUDA;
+  int r = launch_gemm_tc<EPI_PARTIAL>(nullptr, st, mt, &ta, &ta, &tb, p, n_tiles, m_tiles, nullptr);
+  if (r) return r;
+  size_t total = (size_t)M * N;
+  sum_partials<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(scratch, splits, total, y);
+  if (cudaGetLastError() != cudaSuccess) return SPEC_E_CUDA;
+  int stw[4];
+  if (cudaMemcpyAsync(stw, p.status, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return SPEC_E_CUDA;
+  return stw[0] == 0 ? SPEC_OK : SPEC_E_TIMEOUT;
+}
+
+}  // extern "C"

@@ -1,0 +1,153 @@
+"""Parity of the CUDA decode loop with the CPU oracle, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+
+from synthetic import controlled_draft, draw_prompt, draw_weights, get_config
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-4     # max|a-b| / max|b| per row, float32 configuration
+TOL_BF16 = 2e-2     # bf16 configurations
+TIE_GAP = 1e-2      # token mismatches are allowed only where the oracle's top-2 gap is below this
+
+SMALL_BF16 = get_config("c0", name="small_bf16", n_layers=3, d_model=256, n_heads=4, n_kv_heads=2, head_dim=64,
+                        d_ffn=704, vocab=3000, dtype="bf16", seed=21, norm_gain="random", rope_base=1e6)
+SMALL_BF16_D128 = SMALL_BF16.with_(name="small_bf16_d128", n_heads=2, n_kv_heads=2, head_dim=128, n_medusa=4,
+                                   topk=(10, 4, 2, 2), tree_nodes=64, seed=22, vocab=32016)
+
+
+@pytest.fixture(scope="module")
+def torch():
+    t = pytest.importorskip("torch")
+    if not t.cuda.is_available():
+        pytest.skip("no CUDA device")
+    return t
+
+
+def _lockstep(cfg, tol, new_tokens, prompt_len=None, tree_nodes=None, flags=0, **kw):
+    from paper_2503_14153_b200 import build_tree
+    from tests_lockstep import run_lockstep
+    w = draw_weights(cfg)
+    prompt = draw_prompt(cfg, prompt_len)
+    tree = build_tree(cfg.topk, tree_nodes or cfg.tree_nodes)
+    return run_lockstep(cfg, w, tree, prompt, new_tokens, tol, TIE_GAP, flags=flags, **kw)
+
+
+def test_c0_tiny_fp32_full_run(torch):
+    """Configuration 0 end to end: 32-token prompt, 16-node tree, 64 new tokens, float32."""
+    cfg = get_config("c0")
+    rep = _lockstep(cfg, TOL_FP32, cfg.new_tokens, check_kv_every=8)
+    assert len(rep.tokens) >= cfg.new_tokens
+    assert not rep.near_ties, rep.near_ties
+    assert rep.max_logit_err < TOL_FP32 and rep.max_kv_err < TOL_FP32
+
+
+def test_c0_chain_tree_and_single_node_tree(torch):
+    from paper_2503_14153_b200 import chain_tree
+    from tests_lockstep import run_lockstep
+    cfg = get_config("c0")
+    w, prompt = draw_weights(cfg), draw_prompt(cfg)
+    a = run_lockstep(cfg, w, chain_tree(cfg.n_medusa + 1), prompt, 24, TOL_FP32)
+    b = run_lockstep(cfg, w, chain_tree(1), prompt, 24, TOL_FP32)
+    assert a.tokens[:24] == b.tokens[:24]
+    assert b.counts == [1] * len(b.counts)
+
+
+def test_c0_random_gains_and_ragged_prompt(torch):
+    cfg = get_config("c0", norm_gain="random", seed=5)
+    rep = _lockstep(cfg, TOL_FP32, 20, prompt_len=37, tree_nodes=11)
+    assert rep.steps > 0
+
+
+def test_c0_long_prompt_spans_several_prefill_passes(torch):
+    cfg = get_config("c0", seed=6)
+    rep = _lockstep(cfg, TOL_FP32, 12, prompt_len=300, check_kv_every=4)
+    assert rep.max_kv_err < TOL_FP32
+
+
+def test_small_bf16_simple_kernels(torch):
+    from paper_2503_14153_b200 import FLAG_SIMPLE_KERNELS
+    rep = _lockstep(SMALL_BF16, TOL_BF16, 24, prompt_len=45, flags=FLAG_SIMPLE_KERNELS, check_kv_every=6)
+    assert rep.max_logit_err < TOL_BF16
+
+
+def test_small_bf16_tensor_core_path(torch):
+    rep = _lockstep(SMALL_BF16, TOL_BF16, 32, prompt_len=45, check_kv_every=6)
+    assert rep.max_logit_err < TOL_BF16
+
+
+def test_small_bf16_d128_tree64_tensor_core_path(torch):
+    rep = _lockstep(SMALL_BF16_D128, TOL_BF16, 24, prompt_len=150, check_kv_every=6)
+    assert rep.max_logit_err < TOL_BF16
+
+
+def test_controlled_draft_accept_lengths(torch):
+    """Controlled-acceptance draft: rank-0 candidate of head j is the true greedy token with
+    probability p. The stream is unchanged and the accepted lengths match the oracle's."""
+    from oracle.decoder import OracleModel
+    from oracle.spec import OracleSpecDecoder
+    from oracle.tree import chain_tree as o_chain
+    cfg = SMALL_BF16
+    w, prompt = draw_weights(cfg), draw_prompt(cfg, 20)
+    model = OracleModel(cfg, w)
+    stream = OracleSpecDecoder(model, o_chain(1), 200).generate(prompt, 80)[0]
+    uniforms, hit = controlled_draft(cfg, stream, 0.7, 80)
+
+    def ov(i, done):
+        t = uniforms[i, :, :].copy()
+        for j in range(cfg.n_medusa):
+            if hit[i, j] and done + 1 + j < len(stream):
+                t[j, 0] = stream[done + 1 + j]
+        return t
+
+    from paper_2503_14153_b200 import build_tree
+    from tests_lockstep import run_lockstep
+    tree = build_tree(cfg.topk, cfg.tree_nodes)
+    rep = run_lockstep(cfg, w, tree, prompt, 60, TOL_BF16, overrides=lambda i, done: ov(i, done)[:, :max(cfg.topk)],
+                       oracle_model=model)
+    ties = {t[0] for t in rep.near_ties}
+    if not ties:
+        assert rep.tokens[:60] == [int(t) for t in stream[:60]]
+    assert np.mean(rep.counts) > 1.5
+
+
+def test_fragment_truncation(torch):
+    from oracle.decoder import OracleModel
+    from oracle.spec import OracleSpecDecoder
+    from oracle.tree import chain_tree as o_chain
+    cfg = get_config("c0")
+    w, prompt = draw_weights(cfg), draw_prompt(cfg)
+    stream = OracleSpecDecoder(OracleModel(cfg, w), o_chain(1), 200).generate(prompt, 40)[0]
+    frag = int(np.bincount(stream).argmax())
+    rep = _lockstep(cfg, TOL_FP32, 40, frag_token=frag)
+    assert rep.tokens[:40] == [int(t) for t in stream[:40]]
+
+
+def test_typical_acceptance_mode(torch):
+    cfg = get_config("c0")
+    rep = _lockstep(cfg, TOL_FP32, 30, accept_mode=1, typ=(0.3, 0.6, 1.0))
+    assert rep.steps > 0
+
+
+@pytest.mark.parametrize("M,N,K,splits", [(16, 128, 64, 1), (64, 384, 256, 2), (64, 4096, 4096, 3),
+                                          (128, 1000, 704, 2), (32, 200, 128, 1), (256, 512, 512, 4)])
+def test_op_linear_bf16_vs_oracle_matmul(torch, M, N, K, splits):
+    from oracle.numerics import round_bf16
+    from paper_2503_14153_b200 import spec_op_linear
+    rng = np.random.default_rng(M * 7 + N)
+    x = round_bf16(rng.standard_normal((M, K)).astype(np.float32))
+    w = round_bf16((rng.standard_normal((N, K)) * 0.05).astype(np.float32))
+    ref = x @ w.T
+    y = spec_op_linear(torch.from_numpy(x.astype(np.float32)).cuda().to(torch.bfloat16),
+                       torch.from_numpy(w.astype(np.float32)).cuda().to(torch.bfloat16), splits).cpu().numpy()
+    err = np.abs(y - ref).max() / np.abs(ref).max()
+    assert err < 1e-5, err
+
+
+def test_op_linear_fp32_vs_oracle_matmul(torch):
+    from paper_2503_14153_b200 import spec_op_linear
+    rng = np.random.default_rng(3)
+    x, w = rng.standard_normal((13, 688)).astype(np.float32), rng.standard_normal((301, 688)).astype(np.float32)
+    y = spec_op_linear(torch.from_numpy(x).cuda(), torch.from_numpy(w).cuda()).cpu().numpy()
+    ref = x.astype(np.float64) @ w.astype(np.float64).T
+    assert np.abs(y - ref).max() / np.abs(ref).max() < 1e-5
