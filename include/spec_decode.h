@@ -142,6 +142,20 @@ enum { SPEC_Q_KMAX = 0, SPEC_Q_KERNEL_LAUNCHES = 1, SPEC_Q_N_NODES = 2, SPEC_Q_B
        SPEC_Q_ALGO_BYTES_PER_STEP = 4 /* weights + lm_head (twice) + heads, in KiB */ };
 int64_t spec_query(const spec_ctx *ctx, int32_t what);
 
+/* Device time of the five parts of the LAST step, in milliseconds, from events recorded on
+ * the stream at the part boundaries: ms[0] heads + lm_head + top-k, ms[1] tree expansion and
+ * embedding gather, ms[2] verification forward incl. lm_head, ms[3] acceptance, ms[4] KV
+ * compaction (the five parts of the step in Sec. III-B). Synchronises. */
+int spec_last_step_phase_ms(spec_ctx *ctx, float *ms /* HOST [5] */);
+
+/* Per-launch timing of one kernel kind of the verification forward: while `kind` != 0 every
+ * launch of that kernel is bracketed by events, each step ends with a stream synchronise and
+ * the elapsed times accumulate. spec_profile_kernel resets the totals. */
+enum { SPEC_PROFILE_OFF = 0, SPEC_PROFILE_GATE_UP = 1, SPEC_PROFILE_QKV = 2, SPEC_PROFILE_WO = 3,
+       SPEC_PROFILE_DOWN = 4, SPEC_PROFILE_ATTENTION = 5 };
+int spec_profile_kernel(spec_ctx *ctx, int32_t kind);
+int spec_profile_read(spec_ctx *ctx, double *total_ms, int64_t *launches); /* HOST outputs */
+
 /* Debug taps (tests): copy an intermediate of the LAST step to HOST memory. Synchronises.
  * Rows are ordered [sequence][tree node]. */
 enum {

@@ -5,6 +5,7 @@ Follows Sec. III-B: the base model scores every candidate position
 state. float64 arithmetic; for "bf16" models operands are quantised at the fixed points
 named in oracle.numerics.
 """
+from concurrent.futures import ThreadPoolExecutor
 from typing import Dict
 
 import numpy as np
@@ -19,8 +20,12 @@ class OracleModel:
         self.cfg = cfg
         self.q = make_quantiser(cfg.dtype)
         if cfg.dtype == "bf16":
-            self.w = {k: (round_bf16(v).astype(np.float32) if v.ndim == 2 or ".b" in k else v)
-                      for k, v in weights.items()}
+            # weights are bf16 values: round every matrix and head bias once (per tensor, in threads)
+            names = [k for k, v in weights.items() if v.ndim == 2 or ".b" in k]
+            with ThreadPoolExecutor(max_workers=8) as ex:
+                rounded = list(ex.map(lambda k: round_bf16(weights[k]).astype(np.float32), names))
+            self.w = dict(weights)
+            self.w.update(dict(zip(names, rounded)))
         else:
             self.w = dict(weights)
 

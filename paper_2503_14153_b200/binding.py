@@ -16,6 +16,7 @@ _lib = None
 
 FLAG_KEEP_LOGITS = 1
 FLAG_SIMPLE_KERNELS = 2
+PROFILE_OFF, PROFILE_GATE_UP, PROFILE_QKV, PROFILE_WO, PROFILE_DOWN, PROFILE_ATTENTION = range(6)
 
 Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB = 0, 1, 2, 3, 4
 (DBG_TOK, DBG_POS, DBG_LOGITS, DBG_HIDDEN, DBG_ARGMAX, DBG_PATH, DBG_CAND, DBG_SEQLEN, DBG_NEXT_ROOT,
@@ -23,7 +24,7 @@ Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB = 0, 1, 2, 3, 4
 
 EXPORTS = ["spec_workspace_bytes", "spec_create", "spec_prefill", "spec_step", "spec_read_generated",
            "spec_destroy", "spec_last_error", "spec_query", "spec_debug_read", "spec_debug_read_kv",
-           "spec_op_linear"]
+           "spec_op_linear", "spec_last_step_phase_ms", "spec_profile_kernel", "spec_profile_read"]
 
 
 class SpecError(RuntimeError):
@@ -89,6 +90,12 @@ def load_library():
     lib.spec_op_linear.restype = C.c_int
     lib.spec_op_linear.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_void_p, C.c_void_p]
+    lib.spec_last_step_phase_ms.restype = C.c_int
+    lib.spec_last_step_phase_ms.argtypes = [C.c_void_p, C.c_void_p]
+    lib.spec_profile_kernel.restype = C.c_int
+    lib.spec_profile_kernel.argtypes = [C.c_void_p, C.c_int32]
+    lib.spec_profile_read.restype = C.c_int
+    lib.spec_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     _lib = lib
     return lib
 
@@ -233,6 +240,20 @@ class SpecDecoder:
         n = C.c_int32(0)
         self._check(self.lib.spec_read_generated(self._ctx, seq, buf.ctypes.data, max_tokens, C.byref(n)))
         return buf[: min(n.value, max_tokens)].copy()
+
+    def phase_ms(self) -> np.ndarray:
+        """Device milliseconds of the last step's five parts (heads, expand, verify, accept, compact)."""
+        ms = np.zeros(5, dtype=np.float32)
+        self._check(self.lib.spec_last_step_phase_ms(self._ctx, ms.ctypes.data))
+        return ms
+
+    def profile_kernel(self, kind: int):
+        self._check(self.lib.spec_profile_kernel(self._ctx, kind))
+
+    def profile_read(self):
+        ms, n = C.c_double(0.0), C.c_int64(0)
+        self._check(self.lib.spec_profile_read(self._ctx, C.byref(ms), C.byref(n)))
+        return ms.value, n.value
 
     def query(self, what: int) -> int:
         return int(self.lib.spec_query(self._ctx, what))

@@ -119,6 +119,14 @@ struct spec_ctx {
   std::map<std::tuple<const void*, uint64_t, uint64_t, uint32_t>, CUtensorMap> tmaps;
   long long launches = 0;
   bool prefilled = false;
+  // timing: phase boundaries of the last step; optional per-launch timing of one kernel kind
+  cudaEvent_t phase_ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  bool phase_valid = false;
+  int profile_kind = 0;                 // SPEC_PROFILE_*
+  std::vector<cudaEvent_t> prof_ev;     // pairs, reused every step
+  int prof_used = 0;
+  double prof_ms = 0.0;
+  long long prof_launches = 0;
   std::string err = "no error";
 
   int fail(int code, const std::string& msg) { err = msg; return code; }
@@ -253,6 +261,26 @@ size_t carve(spec_ctx* c, void* base) {
     if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string(name) + ": " + cudaGetErrorString(e_)); \
   } while (0)
 
+// Brackets one launch with events when that kernel kind is being profiled.
+struct ProfScope {
+  spec_ctx* c;
+  bool on;
+  ProfScope(spec_ctx* ctx, int kind) : c(ctx), on(ctx->profile_kind == kind && kind != 0) {
+    if (!on) return;
+    if ((size_t)c->prof_used + 2 > c->prof_ev.size()) {
+      cudaEvent_t a, b;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
+      c->prof_ev.push_back(a); c->prof_ev.push_back(b);
+    }
+    cudaEventRecord(c->prof_ev[c->prof_used], c->stream);
+  }
+  ~ProfScope() {
+    if (!on) return;
+    cudaEventRecord(c->prof_ev[c->prof_used + 1], c->stream);
+    c->prof_used += 2;
+  }
+};
+
 Rows make_rows(spec_ctx* c, int R, bool chain) {
   Rows r;
   r.R = R; r.B = c->B;
@@ -288,7 +316,7 @@ int launch_gemm_tc(spec_ctx* c, cudaStream_t st, int mt, const CUtensorMap* a, c
 }
 
 // y partials = x[M,K] W[N,K]^T; returns the number of K slices used (>0) or a negative error.
-int linear_tc_partial(spec_ctx* c, const void* x, const void* W, int M, int N, int K, float* out) {
+int linear_tc_partial(spec_ctx* c, const void* x, const void* W, int M, int N, int K, float* out, int kind) {
   int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (N + 127) / 128;
   int s = splits_for(n_tiles, m_tiles, K);
   if ((size_t)s * M * N > c->part_floats && out == c->d_part) return c->fail(SPEC_E_NOMEM, "split-K scratch too small");
@@ -298,8 +326,11 @@ int linear_tc_partial(spec_ctx* c, const void* x, const void* W, int M, int N, i
   GemmTcParams p{};
   p.M = M; p.N = N; p.K = K; p.splits = s; p.a2_row_offset = 64; p.tile_rows = 128;
   p.out = out; p.split_stride = (size_t)M * N; p.ldo = N; p.status = c->d_status;
-  if (launch_gemm_tc<EPI_PARTIAL>(c, c->stream, mt, ta, ta, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
-    return c->fail(SPEC_E_CUDA, std::string("gemm_tc launch: ") + cudaGetErrorString(cudaGetLastError()));
+  {
+    ProfScope ps(c, kind);
+    if (launch_gemm_tc<EPI_PARTIAL>(c, c->stream, mt, ta, ta, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
+      return c->fail(SPEC_E_CUDA, std::string("gemm_tc launch: ") + cudaGetErrorString(cudaGetLastError()));
+  }
   return s;
 }
 
@@ -333,7 +364,7 @@ int forward_layers(spec_ctx* c, int R, bool chain) {
     int sq = 1;
     if (c->tc) {
       if (c->qkv_fused) {
-        sq = linear_tc_partial(c, u, c->wq[l], M, c->Nqkv, d, c->d_part);
+        sq = linear_tc_partial(c, u, c->wq[l], M, c->Nqkv, d, c->d_part, SPEC_PROFILE_QKV);
         if (sq < 0) return sq;
       } else {
         return c->fail(SPEC_E_BADARG, "bf16 path needs wq/wk/wv contiguous per layer");
@@ -362,6 +393,7 @@ int forward_layers(spec_ctx* c, int R, bool chain) {
         if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_tc<HDV, NWV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); set_ = true; } \
         attention_tc<HDV, NWV><<<grid, NWV * 32, sm, c->stream>>>(a);                                    \
       }
+      ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
       if (D == 128) {
         if (nw <= 1) ATTN_CASE(128, 1) else if (nw <= 2) ATTN_CASE(128, 2) else if (nw <= 4) ATTN_CASE(128, 4) else ATTN_CASE(128, 8)
       } else {
@@ -380,7 +412,7 @@ int forward_layers(spec_ctx* c, int R, bool chain) {
     }
     // output projection + residual + FFN norm
     int so = 1;
-    if (c->tc) { so = linear_tc_partial(c, attn, c->wo[l], M, d, HD, c->d_part); if (so < 0) return so; }
+    if (c->tc) { so = linear_tc_partial(c, attn, c->wo[l], M, d, HD, c->d_part, SPEC_PROFILE_WO); if (so < 0) return so; }
     else { int r = linear_simple<T>(c, attn, HD, static_cast<const T*>(c->wo[l]), c->d_part, d, M, d, HD); if (r) return r; }
     rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, so, (size_t)M * d, c->fn[l], f.rms_eps, u, nullptr, d);
     LAUNCH_CHECK("rmsnorm_rows");
@@ -394,6 +426,7 @@ int forward_layers(spec_ctx* c, int R, bool chain) {
       GemmTcParams p{};
       p.M = M; p.N = F; p.K = d; p.splits = 1; p.a2_row_offset = 0; p.tile_rows = 64;
       p.act = reinterpret_cast<bf16*>(act); p.ld_act = F; p.status = c->d_status;
+      ProfScope ps(c, SPEC_PROFILE_GATE_UP);
       if (launch_gemm_tc<EPI_SWIGLU>(c, c->stream, mt, tg, tu, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
         return c->fail(SPEC_E_CUDA, std::string("gemm_tc swiglu launch: ") + cudaGetErrorString(cudaGetLastError()));
     } else {
@@ -406,7 +439,7 @@ int forward_layers(spec_ctx* c, int R, bool chain) {
       swiglu_rows<T><<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(g, up, act, total);
       LAUNCH_CHECK("swiglu_rows");
     }
-    if (c->tc) { pending = linear_tc_partial(c, act, c->wd[l], M, d, F, c->d_part); if (pending < 0) return pending; }
+    if (c->tc) { pending = linear_tc_partial(c, act, c->wd[l], M, d, F, c->d_part, SPEC_PROFILE_DOWN); if (pending < 0) return pending; }
     else { int r = linear_simple<T>(c, act, F, static_cast<const T*>(c->wd[l]), c->d_part, d, M, d, F); if (r) return r; pending = 1; }
     pending_stride = (size_t)M * d;
   }
@@ -516,6 +549,10 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   int B = c->B, K = c->K, T_ = c->T, d = f.d_model, kmax = c->kmax;
   for (int b = 0; b < B; ++b)
     if (c->n_hi[b] + K + 1 > f.max_seq) return c->fail(SPEC_E_SEQLEN, "sequence would exceed max_seq");
+  for (int i = 0; i < 6; ++i)
+    if (!c->phase_ev[i]) CUDA_OK(cudaEventCreate(&c->phase_ev[i]));
+  c->prof_used = 0;
+  cudaEventRecord(c->phase_ev[0], c->stream);
   const int* ov = nullptr;
   if (cand_override && K > 0) {
     CUDA_OK(cudaMemcpyAsync(c->d_cand_ov, cand_override, (size_t)B * K * kmax * sizeof(int), cudaMemcpyHostToDevice, c->stream));
@@ -541,17 +578,20 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   } else {
     CUDA_OK(cudaMemcpyAsync(c->d_cand, c->d_root, B * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
   }
+  cudaEventRecord(c->phase_ev[1], c->stream);
   // (2) candidate tree -> rows
   int M = B * T_;
   Rows rows = make_rows(c, T_, false);
   prepare_verify_rows<T><<<M, 128, 0, c->stream>>>(rows, c->d_cand, (K + 1) * kmax, kmax, c->d_depth, c->d_rank, c->cap,
                                                  static_cast<const T*>(c->embed), c->d_x, d, f.vocab, c->d_status);
   LAUNCH_CHECK("prepare_verify_rows");
+  cudaEventRecord(c->phase_ev[2], c->stream);
   // (3) verification forward
   int r = forward_layers<T>(c, T_, false);
   if (r) return r;
   r = lm_head_argmax<T>(c, static_cast<const T*>(c->d_hq), M);
   if (r) return r;
+  cudaEventRecord(c->phase_ev[3], c->stream);
   // (4) acceptance
   AcceptArgs a = make_accept(c, T_, 0);
   if (f.accept_mode == 1) {
@@ -562,10 +602,20 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   }
   accept_kernel<<<B, 128, 0, c->stream>>>(a);
   LAUNCH_CHECK("accept_kernel");
+  cudaEventRecord(c->phase_ev[4], c->stream);
   // (5) KV compaction
   dim3 gc(f.n_layers * 2 * f.n_kv_heads, B);
   compact_kv<T><<<gc, 64, 0, c->stream>>>(static_cast<T*>(c->d_pool), c->geom, c->d_page_table, c->d_path, c->d_count, c->d_n_old, K);
   LAUNCH_CHECK("compact_kv");
+  cudaEventRecord(c->phase_ev[5], c->stream);
+  c->phase_valid = true;
+  if (c->profile_kind) {
+    CUDA_OK(cudaStreamSynchronize(c->stream));
+    for (int i = 0; i + 1 < c->prof_used; i += 2) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]) == cudaSuccess) { c->prof_ms += ms; c->prof_launches++; }
+    }
+  }
   if (out_tokens || out_counts) {
     if (out_tokens) CUDA_OK(cudaMemcpyAsync(out_tokens, c->d_out_tok, (size_t)B * (K + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
     if (out_counts) CUDA_OK(cudaMemcpyAsync(out_counts, c->d_count, (size_t)B * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
@@ -718,6 +768,8 @@ int spec_read_generated(spec_ctx* c, int32_t seq, int32_t* out, int32_t max_toke
 int spec_destroy(spec_ctx* c) {
   if (!c) return SPEC_E_BADARG;
   cudaStreamSynchronize(c->stream);
+  for (int i = 0; i < 6; ++i) if (c->phase_ev[i]) cudaEventDestroy(c->phase_ev[i]);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c;
   return SPEC_OK;
 }
@@ -740,6 +792,29 @@ int64_t spec_query(const spec_ctx* c, int32_t what) {
     }
     default: return -1;
   }
+}
+
+int spec_last_step_phase_ms(spec_ctx* c, float* ms) {
+  if (!c || !ms) return SPEC_E_BADARG;
+  if (!c->phase_valid) return c->fail(SPEC_E_STATE, "no step has run");
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  for (int i = 0; i < 5; ++i) CUDA_OK(cudaEventElapsedTime(&ms[i], c->phase_ev[i], c->phase_ev[i + 1]));
+  return SPEC_OK;
+}
+
+int spec_profile_kernel(spec_ctx* c, int32_t kind) {
+  if (!c || kind < 0 || kind > SPEC_PROFILE_ATTENTION) return SPEC_E_BADARG;
+  c->profile_kind = kind;
+  c->prof_ms = 0.0;
+  c->prof_launches = 0;
+  return SPEC_OK;
+}
+
+int spec_profile_read(spec_ctx* c, double* total_ms, int64_t* launches) {
+  if (!c || !total_ms || !launches) return SPEC_E_BADARG;
+  *total_ms = c->prof_ms;
+  *launches = c->prof_launches;
+  return SPEC_OK;
 }
 
 int spec_debug_read(spec_ctx* c, int32_t what, void* host_buf, size_t bytes) {

@@ -7,3 +7,4 @@ neither the oracle nor the CUDA binding.
 from .configs import ModelConfig, CONFIGS, get_config  # noqa: F401
 from .weights import tensor_specs, draw_tensor, draw_weights  # noqa: F401
 from .prompts import draw_prompt, draw_prompt_batch, controlled_draft  # noqa: F401
+from .device import stream_weights_to_device  # noqa: F401
