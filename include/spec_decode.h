@@ -190,6 +190,25 @@ int spec_debug_read_kv(spec_ctx *ctx, int32_t seq, int32_t layer, int32_t slot0,
 int spec_op_linear(int32_t dtype, const void *x, const void *w, float *y, int32_t M, int32_t N,
                    int32_t K, int32_t splits, float *scratch, void *cuda_stream);
 
+/* The same operation as spec_op_linear for callers that cannot allocate device memory and so
+ * have no scratch buffer to pass: code running where cudaMalloc is forbidden (inside a
+ * real-time or safety-certified loop, under a framework whose memory pool is frozen or
+ * exhausted, in a plug-in that was handed only its input and output buffers). The paper has no
+ * counterpart; this entry exists for those callers only.
+ * The K-slice partial sums and the status word live in an array built into the library
+ * (SPEC_STATIC_SCRATCH_FLOATS float32 values, 8 MiB, held by every GPU that loads the library
+ * until the process exits). A call with splits*M*N above that limit returns SPEC_E_NOMEM and
+ * spec_last_error(NULL) says by how much. The call itself allocates nothing, on host or device.
+ * The first call on each device looks the array's device address up (with that device
+ * current) and keeps it; make that first call outside any stream capture. All calls share the
+ * one array: it still holds the previous call's partial sums (the library clears the status
+ * word itself), and two calls whose kernels overlap on the GPU - different streams, or
+ * different host threads - race on it. Serialise them.
+ * Arguments, limits, results and synchronisation are those of spec_op_linear. */
+#define SPEC_STATIC_SCRATCH_FLOATS (2u << 20)
+int spec_op_linear_static(int32_t dtype, const void *x, const void *w, float *y, int32_t M, int32_t N,
+                          int32_t K, int32_t splits, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,8 @@ Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB = 0, 1, 2, 3, 4
 
 EXPORTS = ["spec_workspace_bytes", "spec_create", "spec_prefill", "spec_step", "spec_read_generated",
            "spec_destroy", "spec_last_error", "spec_query", "spec_debug_read", "spec_debug_read_kv",
-           "spec_op_linear", "spec_last_step_phase_ms", "spec_profile_kernel", "spec_profile_read"]
+           "spec_op_linear", "spec_op_linear_static", "spec_last_step_phase_ms", "spec_profile_kernel",
+           "spec_profile_read"]
 
 
 class SpecError(RuntimeError):
@@ -90,6 +91,9 @@ def load_library():
     lib.spec_op_linear.restype = C.c_int
     lib.spec_op_linear.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_void_p, C.c_void_p]
+    lib.spec_op_linear_static.restype = C.c_int
+    lib.spec_op_linear_static.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                          C.c_int32, C.c_int32, C.c_void_p]
     lib.spec_last_step_phase_ms.restype = C.c_int
     lib.spec_last_step_phase_ms.argtypes = [C.c_void_p, C.c_void_p]
     lib.spec_profile_kernel.restype = C.c_int
@@ -292,4 +296,24 @@ def spec_op_linear(x, w, splits: int = 1):
                             torch.cuda.current_stream(x.device).cuda_stream)
     if rc != 0:
         raise SpecError(rc, "spec_op_linear failed")
+    return y
+
+
+STATIC_SCRATCH_FLOATS = 2 << 20
+
+
+def spec_op_linear_static(x, w, y, splits: int = 1):
+    """y[M,N] (float32, preallocated by the caller) = x @ w.T through the entry point that keeps
+    its scratch inside the library. For callers that may not allocate device memory: nothing
+    is allocated here either, the three tensors are used as given. Raises SpecError with the
+    library's message when splits*M*N exceeds STATIC_SCRATCH_FLOATS."""
+    import torch
+    lib = load_library()
+    M, K = x.shape
+    N = w.shape[0]
+    dtype = 1 if x.dtype == torch.bfloat16 else 0
+    rc = lib.spec_op_linear_static(dtype, x.data_ptr(), w.data_ptr(), y.data_ptr(), M, N, K, splits,
+                                   torch.cuda.current_stream(x.device).cuda_stream)
+    if rc != 0:
+        raise SpecError(rc, lib.spec_last_error(None).decode())
     return y

@@ -913,4 +913,66 @@ int spec_op_linear(int32_t dtype, const void* x, const void* w, float* y, int32_
   return stw[0] == 0 ? SPEC_OK : SPEC_E_TIMEOUT;
 }
 
+
+// ---- the linear operation for callers that cannot allocate device memory ----
+// The K-slice partial sums and the status word of spec_op_linear_static live here instead of in
+// a caller-provided buffer. Every context that loads the library holds these bytes until exit.
+static __device__ __align__(256) float g_static_linear_scratch[SPEC_STATIC_SCRATCH_FLOATS + 4];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
+}  // namespace
+
+int spec_op_linear_static(int32_t dtype, const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                          int32_t splits, void* cuda_stream) {
+  if (!x || !w || !y || M < 1 || N < 1 || K < 8 || K % 8 || M > 2048) { g_create_error = "spec_op_linear_static: bad argument"; return SPEC_E_BADARG; }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (dtype == 0) {
+    constexpr int MC = 8;
+    dim3 grid((N + 7) / 8, (M + MC - 1) / MC);
+    linear_rows<float, MC><<<grid, 256, 0, st>>>(static_cast<const float*>(x), K, static_cast<const float*>(w), y, N, M, N, K);
+    return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_E_CUDA;
+  }
+  if (dtype != 1 || K % 64 || splits < 1 || splits > K / 64 || M % 16) { g_create_error = "spec_op_linear_static: bad argument"; return SPEC_E_BADARG; }
+  if ((size_t)splits * M * N > (size_t)SPEC_STATIC_SCRATCH_FLOATS) {
+    char buf[160];
+    snprintf(buf, sizeof(buf), "spec_op_linear_static: splits*M*N = %zu floats exceeds the built-in scratch of %u floats",
+             (size_t)splits * M * N, (unsigned)SPEC_STATIC_SCRATCH_FLOATS);
+    g_create_error = buf;
+    return SPEC_E_NOMEM;
+  }
+  // Set-up, once per device: the array's name is only a host-side handle here, so ask the
+  // runtime for its address on the current device and keep it.
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { g_create_error = "spec_op_linear_static: cudaGetDevice failed"; return SPEC_E_CUDA; }
+  float* scratch = g_static_scratch_addr[dev];
+  if (!scratch) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_linear_scratch);
+    if (e != cudaSuccess || !p) { g_create_error = std::string("spec_op_linear_static: cudaGetSymbolAddress: ") + cudaGetErrorString(e); return SPEC_E_CUDA; }
+    scratch = static_cast<float*>(p);
+    g_static_scratch_addr[dev] = scratch;
+  }
+  int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (N + 127) / 128;
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, w, N, K, 64) || !make_tmap(&tb, x, M, K, mt)) { g_create_error = "spec_op_linear_static: cuTensorMapEncodeTiled failed"; return SPEC_E_CUDA; }
+  GemmTcParams p{};
+  p.M = M; p.N = N; p.K = K; p.splits = splits; p.a2_row_offset = 64; p.tile_rows = 128;
+  p.out = scratch; p.split_stride = (size_t)M * N; p.ldo = N;
+  p.status = reinterpret_cast<int*>(scratch + (size_t)SPEC_STATIC_SCRATCH_FLOATS);
+  // the array keeps the previous call's contents: the status word must start at zero (the
+  // partial sums are fully overwritten before they are read)
+  if (cudaMemsetAsync(p.status, 0, 16, st) != cudaSuccess) return SPEC_E_CUDA;
+  int r = launch_gemm_tc<EPI_PARTIAL>(nullptr, st, mt, &ta, &ta, &tb, p, n_tiles, m_tiles, nullptr);
+  if (r) return r;
+  size_t total = (size_t)M * N;
+  sum_partials<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(scratch, splits, total, y);
+  if (cudaGetLastError() != cudaSuccess) return SPEC_E_CUDA;
+  int stw[4];
+  if (cudaMemcpyAsync(stw, p.status, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return SPEC_E_CUDA;
+  return stw[0] == 0 ? SPEC_OK : SPEC_E_TIMEOUT;
+}
+
 }  // extern "C"
