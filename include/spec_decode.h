@@ -99,9 +99,8 @@ size_t spec_workspace_bytes(const spec_config *cfg, const spec_tree *tree);
 /* Builds a context. `workspace` is a DEVICE buffer of at least spec_workspace_bytes(),
  * 1024-byte aligned, zero-filled or not (the library initialises what it needs).
  * `cuda_stream` is a cudaStream_t (NULL = default stream); all work is enqueued on it.
- * If the q/k/v matrices of a layer are one contiguous allocation in the order wq, wk, wv
- * (wk[l] == wq[l] + n_heads*head_dim*d_model elements, and so on) the three projections
- * run as one launch; otherwise as three.
+ * The q, k and v projections of a layer run as one launch (bf16) whether or not the three
+ * matrices are one allocation.
  * Config and tree are copied; weights, workspace and stream are borrowed. */
 int spec_create(const spec_config *cfg, const spec_weights *weights, const spec_tree *tree,
                 void *workspace, size_t workspace_bytes, void *cuda_stream, spec_ctx **out);
@@ -141,6 +140,16 @@ const char *spec_last_error(const spec_ctx *ctx);
 enum { SPEC_Q_KMAX = 0, SPEC_Q_KERNEL_LAUNCHES = 1, SPEC_Q_N_NODES = 2, SPEC_Q_BATCH = 3,
        SPEC_Q_ALGO_BYTES_PER_STEP = 4 /* weights + lm_head (twice) + heads, in KiB */ };
 int64_t spec_query(const spec_ctx *ctx, int32_t what);
+
+/* Tuning knobs of a context (defaults in brackets). SPEC_OPT_PDL [1]: launch the kernels of
+ * a step with programmatic dependent launch, so that each kernel's set-up and weight prefetch
+ * overlap the tail of the one before. SPEC_OPT_GEMM_CTAS [296]: persistent CTAs the
+ * weight-streaming GEMM deals its work to (1..296). SPEC_OPT_L2_PREFETCH [8]: 16 KiB weight
+ * chunks each GEMM CTA requests into L2, beyond its shared-memory ring, before it waits for the
+ * previous kernel (0..64). Results do not depend on SPEC_OPT_PDL or SPEC_OPT_L2_PREFETCH;
+ * SPEC_OPT_GEMM_CTAS changes the order in which partial sums are added. */
+enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2 };
+int spec_set_option(spec_ctx *ctx, int32_t what, int32_t value);
 
 /* Device time of the five parts of the LAST step, in milliseconds, from events recorded on
  * the stream at the part boundaries: ms[0] heads + lm_head + top-k, ms[1] tree expansion and
@@ -182,23 +191,26 @@ int spec_debug_read_kv(spec_ctx *ctx, int32_t seq, int32_t layer, int32_t slot0,
 
 /* y[M,N] (float32, DEVICE) = x[M,K] * W[N,K]^T for DEVICE x and W of type `dtype`
  * (Sec. III-B verification forward: every projection of the base model). bf16 runs the
- * tensor-core weight-streaming kernel with `splits` K-slices whose float32 partial sums
- * are written to `scratch` (DEVICE, splits*M*N + 4 floats; the last four hold the call's
- * status word) and then summed into y in slice order; float32 runs the CUDA-core row kernel
- * (splits and scratch ignored). M <= 2048; for bf16 K % 64 == 0 and M % 16 == 0.
+ * tensor-core weight-streaming kernel: the (128-row weight tile, 64-wide K chunk) units are
+ * dealt in equal contiguous runs to `ctas` persistent CTAs, runs that end inside a tile leave
+ * float32 partial sums in `scratch` (DEVICE, spec_op_linear_scratch_floats() + 4 floats; the
+ * last four hold the call's status word) and a second kernel adds a tile's partial sums in CTA
+ * order into y. float32 runs the CUDA-core row kernel (ctas and scratch ignored).
+ * M <= 2048; for bf16 K % 64 == 0, M % 16 == 0, N >= 128, 1 <= ctas <= 1024.
  * Synchronises in bf16 mode. */
+size_t spec_op_linear_scratch_floats(int32_t M, int32_t N, int32_t K, int32_t ctas);
 int spec_op_linear(int32_t dtype, const void *x, const void *w, float *y, int32_t M, int32_t N,
-                   int32_t K, int32_t splits, float *scratch, void *cuda_stream);
+                   int32_t K, int32_t ctas, float *scratch, void *cuda_stream);
 
 /* The same operation as spec_op_linear for callers that cannot allocate device memory and so
  * have no scratch buffer to pass: code running where cudaMalloc is forbidden (inside a
  * real-time or safety-certified loop, under a framework whose memory pool is frozen or
  * exhausted, in a plug-in that was handed only its input and output buffers). The paper has no
  * counterpart; this entry exists for those callers only.
- * The K-slice partial sums and the status word live in an array built into the library
+ * The partial sums and the status word live in an array built into the library
  * (SPEC_STATIC_SCRATCH_FLOATS float32 values, 8 MiB, held by every GPU that loads the library
- * until the process exits). A call with splits*M*N above that limit returns SPEC_E_NOMEM and
- * spec_last_error(NULL) says by how much. The call itself allocates nothing, on host or device.
+ * until the process exits). A call that needs more than that (spec_op_linear_scratch_floats()
+ * says how much a shape needs) returns SPEC_E_NOMEM and spec_last_error(NULL) says by how much. The call itself allocates nothing, on host or device.
  * The first call on each device looks the array's device address up (with that device
  * current) and keeps it; make that first call outside any stream capture. All calls share the
  * one array: it still holds the previous call's partial sums (the library clears the status
@@ -207,7 +219,7 @@ int spec_op_linear(int32_t dtype, const void *x, const void *w, float *y, int32_
  * Arguments, limits, results and synchronisation are those of spec_op_linear. */
 #define SPEC_STATIC_SCRATCH_FLOATS (2u << 20)
 int spec_op_linear_static(int32_t dtype, const void *x, const void *w, float *y, int32_t M, int32_t N,
-                          int32_t K, int32_t splits, void *cuda_stream);
+                          int32_t K, int32_t ctas, void *cuda_stream);
 
 #ifdef __cplusplus
 }

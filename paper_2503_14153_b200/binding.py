@@ -19,12 +19,13 @@ FLAG_SIMPLE_KERNELS = 2
 PROFILE_OFF, PROFILE_GATE_UP, PROFILE_QKV, PROFILE_WO, PROFILE_DOWN, PROFILE_ATTENTION = range(6)
 
 Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB = 0, 1, 2, 3, 4
+OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH = 0, 1, 2
 (DBG_TOK, DBG_POS, DBG_LOGITS, DBG_HIDDEN, DBG_ARGMAX, DBG_PATH, DBG_CAND, DBG_SEQLEN, DBG_NEXT_ROOT,
  DBG_H_LAST, DBG_STATUS) = range(11)
 
 EXPORTS = ["spec_workspace_bytes", "spec_create", "spec_prefill", "spec_step", "spec_read_generated",
            "spec_destroy", "spec_last_error", "spec_query", "spec_debug_read", "spec_debug_read_kv",
-           "spec_op_linear", "spec_op_linear_static", "spec_last_step_phase_ms", "spec_profile_kernel",
+           "spec_op_linear", "spec_op_linear_scratch_floats", "spec_op_linear_static", "spec_set_option", "spec_last_step_phase_ms", "spec_profile_kernel",
            "spec_profile_read"]
 
 
@@ -91,6 +92,10 @@ def load_library():
     lib.spec_op_linear.restype = C.c_int
     lib.spec_op_linear.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_void_p, C.c_void_p]
+    lib.spec_op_linear_scratch_floats.restype = C.c_size_t
+    lib.spec_op_linear_scratch_floats.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32]
+    lib.spec_set_option.restype = C.c_int
+    lib.spec_set_option.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
     lib.spec_op_linear_static.restype = C.c_int
     lib.spec_op_linear_static.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_void_p]
@@ -259,6 +264,9 @@ class SpecDecoder:
         self._check(self.lib.spec_profile_read(self._ctx, C.byref(ms), C.byref(n)))
         return ms.value, n.value
 
+    def set_option(self, what: int, value: int):
+        self._check(self.lib.spec_set_option(self._ctx, what, value))
+
     def query(self, what: int) -> int:
         return int(self.lib.spec_query(self._ctx, what))
 
@@ -282,7 +290,7 @@ class SpecDecoder:
         return k, v
 
 
-def spec_op_linear(x, w, splits: int = 1):
+def spec_op_linear(x, w, ctas: int = 296):
     """y = x @ w.T through the library's linear kernel (x, w: CUDA tensors, float32 or bf16)."""
     import torch
     lib = load_library()
@@ -290,8 +298,13 @@ def spec_op_linear(x, w, splits: int = 1):
     N = w.shape[0]
     dtype = 1 if x.dtype == torch.bfloat16 else 0
     y = torch.empty((M, N), dtype=torch.float32, device=x.device)
-    scratch = torch.empty(splits * M * N + 4, dtype=torch.float32, device=x.device) if dtype == 1 else None
-    rc = lib.spec_op_linear(dtype, x.data_ptr(), w.data_ptr(), y.data_ptr(), M, N, K, splits,
+    scratch = None
+    if dtype == 1:
+        need = int(lib.spec_op_linear_scratch_floats(M, N, K, ctas))
+        if need == 0:
+            raise SpecError(-1, "spec_op_linear_scratch_floats rejected the shape")
+        scratch = torch.empty(need + 4, dtype=torch.float32, device=x.device)
+    rc = lib.spec_op_linear(dtype, x.data_ptr(), w.data_ptr(), y.data_ptr(), M, N, K, ctas,
                             scratch.data_ptr() if scratch is not None else None,
                             torch.cuda.current_stream(x.device).cuda_stream)
     if rc != 0:
@@ -302,17 +315,17 @@ def spec_op_linear(x, w, splits: int = 1):
 STATIC_SCRATCH_FLOATS = 2 << 20
 
 
-def spec_op_linear_static(x, w, y, splits: int = 1):
+def spec_op_linear_static(x, w, y, ctas: int = 296):
     """y[M,N] (float32, preallocated by the caller) = x @ w.T through the entry point that keeps
     its scratch inside the library. For callers that may not allocate device memory: nothing
     is allocated here either, the three tensors are used as given. Raises SpecError with the
-    library's message when splits*M*N exceeds STATIC_SCRATCH_FLOATS."""
+    library's message when the shape needs more than STATIC_SCRATCH_FLOATS of partial sums."""
     import torch
     lib = load_library()
     M, K = x.shape
     N = w.shape[0]
     dtype = 1 if x.dtype == torch.bfloat16 else 0
-    rc = lib.spec_op_linear_static(dtype, x.data_ptr(), w.data_ptr(), y.data_ptr(), M, N, K, splits,
+    rc = lib.spec_op_linear_static(dtype, x.data_ptr(), w.data_ptr(), y.data_ptr(), M, N, K, ctas,
                                    torch.cuda.current_stream(x.device).cuda_stream)
     if rc != 0:
         raise SpecError(rc, lib.spec_last_error(None).decode())

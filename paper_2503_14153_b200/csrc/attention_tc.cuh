@@ -58,6 +58,8 @@ attention_tc(const AttnTcArgs a) {
   uint8_t* vs = ks + 2 * TILE_BYTES;                        // [2][KT][HD]
   uint64_t* full = reinterpret_cast<uint64_t*>(vs + 2 * TILE_BYTES);   // [2]
 
+  pdl_launch_dependents();
+  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int h = blockIdx.x, sp = blockIdx.y, b = blockIdx.z;
   const int R = a.rows.R, cnt = a.rows.cnt[b], n = a.rows.n[b];
@@ -235,6 +237,8 @@ attention_tc(const AttnTcArgs a) {
 // w_s = 2^(m_s - max_s m_s). One thread per (row, head, 4 dims).
 __global__ void attention_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml, int nsplit,
                                   Rows rows, int H, int HD, bf16* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
   int M = rows.B * rows.R;
   size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   size_t per_row = (size_t)H * HD / 4;

@@ -366,9 +366,9 @@ __global__ void typical_edges(const float* __restrict__ logits, int V, Rows rows
 // ------------------------------------------------------------------ acceptance walk
 struct AcceptArgs {
   Rows rows;
-  const float* pval;   // [ntile][pstride]
+  const float* pval;   // [row][ntile]
   const int* pidx;
-  int ntile, pstride;
+  int ntile;
   const int *parent, *depth;   // tree arrays [R]
   const int* edge_ok;          // typical mode: per-row pass flag; NULL = greedy token match
   int K, frag_token, d, mode;  // mode 0 = verify step, 1 = prefill (row b is sequence b)
@@ -378,36 +378,50 @@ struct AcceptArgs {
   int *gen_log, *gen_cnt, gen_cap;
 };
 
-// One block per sequence: finishes the per-node argmax from the per-tile partials, walks the
-// tree (a node is accepted iff its parent is and its token is the argmax at the parent, or
-// its Eq. 1 flag is set), takes the deepest accepted node (lowest index on ties), applies
-// the fragment-integrity rule, and publishes the step's result and the next step's state.
-__global__ void accept_kernel(AcceptArgs a) {
-  int b = blockIdx.x, R = a.rows.R;
-  __shared__ int am_s[SPEC_MAX_NODES];
+// One block per sequence: finishes the per-node argmax from the partials (pval/pidx
+// [row][ntile], a warp per row), walks the tree (a node is accepted iff its parent is and its
+// token is the argmax at the parent, or its Eq. 1 flag is set), takes the deepest accepted node
+// (lowest index on ties), applies the fragment-integrity rule, and publishes the step's result
+// and the next step's state.
+__global__ void __launch_bounds__(256) accept_kernel(AcceptArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.x, R = a.rows.R;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  __shared__ int am_s[SPEC_MAX_NODES], tok_s[SPEC_MAX_NODES], par_s[SPEC_MAX_NODES], dep_s[SPEC_MAX_NODES];
   __shared__ int last_s, len_s;
   if (a.mode == 1) {
-    if (threadIdx.x == 0) {
+    if (warp == 0) {
       float bv = -INFINITY; int bi = 0x7fffffff;
-      for (int t = 0; t < a.ntile; ++t) {
-        float v = a.pval[(size_t)t * a.pstride + b]; int i = a.pidx[(size_t)t * a.pstride + b];
+      for (int t = lane; t < a.ntile; t += 32) {
+        float v = a.pval[(size_t)b * a.ntile + t]; int i = a.pidx[(size_t)b * a.ntile + t];
         if (better(v, i, bv, bi)) { bv = v; bi = i; }
       }
-      a.am[b] = bi;
-      a.root_tok[b] = bi;
-      a.gen_cnt[b] = 0;
+      warp_argmax(bv, bi);
+      if (lane == 0) {
+        a.am[b] = bi;
+        a.root_tok[b] = bi;
+        a.gen_cnt[b] = 0;
+      }
     }
     return;
   }
-  int cnt = a.rows.cnt[b], m0 = b * R;
-  for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+  const int cnt = a.rows.cnt[b], m0 = b * R;
+  for (int i = warp; i < cnt; i += nw) {
     float bv = -INFINITY; int bi = 0x7fffffff;
-    for (int t = 0; t < a.ntile; ++t) {
-      float v = a.pval[(size_t)t * a.pstride + m0 + i]; int idx = a.pidx[(size_t)t * a.pstride + m0 + i];
+    const float* pv = a.pval + (size_t)(m0 + i) * a.ntile;
+    const int* pi = a.pidx + (size_t)(m0 + i) * a.ntile;
+    for (int t = lane; t < a.ntile; t += 32) {
+      float v = pv[t]; int idx = pi[t];
       if (better(v, idx, bv, bi)) { bv = v; bi = idx; }
     }
-    am_s[i] = bi;
-    a.am[m0 + i] = bi;
+    warp_argmax(bv, bi);
+    if (lane == 0) { am_s[i] = bi; a.am[m0 + i] = bi; }
+  }
+  for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+    tok_s[i] = a.rows.tok[m0 + i];
+    par_s[i] = a.parent[i];
+    dep_s[i] = a.depth[i];
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -418,25 +432,25 @@ __global__ void accept_kernel(AcceptArgs a) {
       uint32_t acc[4] = {1u, 0u, 0u, 0u};
       int best = 0;
       for (int v = 1; v < cnt; ++v) {
-        int p = a.parent[v];
+        int p = par_s[v];
         bool ok = (acc[p >> 5] >> (p & 31)) & 1u;
-        if (ok) ok = a.edge_ok ? (a.edge_ok[m0 + v] != 0) : (a.rows.tok[m0 + v] == am_s[p]);
+        if (ok) ok = a.edge_ok ? (a.edge_ok[m0 + v] != 0) : (tok_s[v] == am_s[p]);
         if (ok) {
           acc[v >> 5] |= 1u << (v & 31);
-          if (a.depth[v] > a.depth[best]) best = v;
+          if (dep_s[v] > dep_s[best]) best = v;
         }
       }
-      len = a.depth[best] + 1;
+      len = dep_s[best] + 1;
       int path[SPEC_MAX_HEADS + 1];
-      for (int u = best; u >= 0; u = a.parent[u]) path[a.depth[u]] = u;
+      for (int u = best; u >= 0; u = par_s[u]) path[dep_s[u]] = u;
       if (a.frag_token >= 0) {
         int keep = 1;
-        for (int j = 0; j < len; ++j) if (a.rows.tok[m0 + path[j]] == a.frag_token) keep = j + 1;
+        for (int j = 0; j < len; ++j) if (tok_s[path[j]] == a.frag_token) keep = j + 1;
         len = keep;
       }
       int n = a.rows.n[b], gc = a.gen_cnt[b];
       for (int j = 0; j < len; ++j) {
-        int t = a.rows.tok[m0 + path[j]];
+        int t = tok_s[path[j]];
         a.path[b * (a.K + 1) + j] = path[j];
         a.out_tok[b * (a.K + 1) + j] = t;
         if (gc + j < a.gen_cap) a.gen_log[(size_t)b * a.gen_cap + gc + j] = t;

@@ -18,7 +18,8 @@
 
 #include "attention_tc.cuh"
 #include "common.cuh"
-#include "gemm_tc.cuh"
+#include "gemm_stream.cuh"
+#include "glue_tc.cuh"
 #include "kernels_simple.cuh"
 
 using namespace spec;
@@ -80,13 +81,86 @@ int mt_for_rows(int M) {
   if (M <= 64) return 64;
   return 128;
 }
-int splits_for(int n_tiles, int m_tiles, int K) {
-  int kc = K / 64;
-  int s = SM_SLOTS / (n_tiles * m_tiles);
-  if (s > 12) s = 12;
-  if (s > kc / 2) s = kc / 2;
-  if (s < 1) s = 1;
-  return s;
+
+// Launch with or without the programmatic-dependent-launch attribute.
+template <typename... Params, typename... Args>
+cudaError_t launch_k(bool pdl, void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+// One launch of the weight-streaming GEMM: shapes, the dealing of units to CTAs and the view
+// of its partial sums.
+struct GemmPlan {
+  StreamGemmParams p;
+  int MT, grid;
+};
+
+bool plan_gemm(int M, int K, int n_mats, const int* rows, int g_max, bool tile_granular, GemmPlan* out) {
+  if (M < 1 || K < 64 || K % 64 || n_mats < 1 || n_mats > GS_MAX_MATS || g_max < 1) return false;
+  GemmPlan& g = *out;
+  g = GemmPlan{};
+  StreamGemmParams& p = g.p;
+  g.MT = mt_for_rows(M);
+  p.M = M; p.K = K; p.n_mats = n_mats;
+  int tiles = 0, col = 0;
+  for (int i = 0; i < n_mats; ++i) {
+    if (rows[i] < 1) return false;
+    p.mat_tile0[i] = tiles; p.mat_rows[i] = rows[i]; p.mat_col0[i] = col;
+    tiles += (rows[i] + 127) / 128;
+    col += rows[i];
+  }
+  for (int i = n_mats; i <= GS_MAX_MATS; ++i) p.mat_tile0[i] = tiles;
+  p.n_tiles = tiles;
+  p.seg.KC = K / 64;
+  p.seg.m_tiles = (M + g.MT - 1) / g.MT;
+  long long total = (long long)tiles * p.seg.m_tiles * p.seg.KC;
+  if (total > 0x3fffffff) return false;
+  p.seg.total = (int)total;
+  p.tile_granular = tile_granular ? 1 : 0;
+  long long cap = tile_granular ? (long long)tiles * p.seg.m_tiles : total;
+  g.grid = (int)std::min<long long>(g_max, cap);
+  p.seg.G = g.grid;
+  return true;
+}
+
+// Upper bound of the partial-sum slots a tile can have when the units go to at most g_max CTAs.
+int plan_slot_bound(const GemmPlan& g) {
+  const SegMap& s = g.p.seg;
+  return (int)(((long long)s.KC * s.G) / s.total) + 2;
+}
+
+size_t plan_part_floats(const GemmPlan& g) { return (size_t)plan_slot_bound(g) * g.p.M * g.p.n_tiles * 128; }
+
+template <int MT>
+cudaError_t launch_gs_mt(cudaStream_t st, bool pdl, int grid, const StreamTmaps& tm, const StreamGemmParams& p) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_stream<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamCfg<MT>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  return launch_k(pdl, gemm_stream<MT>, dim3(grid), dim3(192), (size_t)StreamCfg<MT>::SMEM_BYTES, st, tm, p);
+}
+cudaError_t launch_gs(cudaStream_t st, bool pdl, const GemmPlan& g, const StreamTmaps& tm) {
+  switch (g.MT) {
+    case 16: return launch_gs_mt<16>(st, pdl, g.grid, tm, g.p);
+    case 32: return launch_gs_mt<32>(st, pdl, g.grid, tm, g.p);
+    case 64: return launch_gs_mt<64>(st, pdl, g.grid, tm, g.p);
+    default: return launch_gs_mt<128>(st, pdl, g.grid, tm, g.p);
+  }
+}
+
+PartView plan_view(const GemmPlan& g) {
+  PartView v{};
+  v.part = g.p.part; v.slot_stride = g.p.slot_stride; v.ld = g.p.n_tiles * 128; v.seg = g.p.seg; v.MT = g.MT;
+  return v;
 }
 
 }  // namespace
@@ -99,6 +173,9 @@ struct spec_ctx {
   size_t esz;                          // operand element size
   int Mcap, cap, pages_per_seq, gen_cap, nsplit_attn, Nqkv, ntile_lm, topk_slice, topk_blocks;
   bool qkv_fused, keep_logits;
+  bool pdl = true;                     // programmatic dependent launch between the kernels of a step
+  int gemm_ctas = SM_SLOTS;            // persistent CTAs of the weight-streaming GEMM
+  int l2_prefetch = 8;                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
   std::vector<int> h_parent, h_depth, h_rank;
   std::vector<int> n_hi;               // host upper bound of committed lengths
   std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, mw, mb;
@@ -174,6 +251,7 @@ bool validate_config(const spec_config* c, std::string* why) {
     if (c->d_model % 64 || c->d_ffn % 64 || (c->n_heads * c->head_dim) % 64) { *why = "bf16 path needs widths that are multiples of 64"; return false; }
     if (c->head_dim != 64 && c->head_dim != 128) { *why = "bf16 path needs head_dim 64 or 128"; return false; }
     if (c->page_size != 16) { *why = "bf16 path needs page_size 16"; return false; }
+    if (c->d_model < 128 || c->d_ffn < 128 || c->vocab < 128 || c->n_kv_heads * c->head_dim < 128) { *why = "bf16 path needs every weight matrix to have at least 128 rows"; return false; }
   } else if (c->dtype == 1 && c->head_dim % 64) { *why = "bf16 cache needs head_dim multiple of 64"; return false; }
   return true;
 }
@@ -190,7 +268,7 @@ size_t carve(spec_ctx* c, void* base) {
   if (64 % f.page_size == 0) c->cap = (int)round_up(c->cap, 64);   // whole 64-key attention tiles
   c->pages_per_seq = c->cap / f.page_size;
   c->gen_cap = f.max_seq + K + 1;
-  c->ntile_lm = c->tc ? (V + 127) / 128 : 1;
+  c->ntile_lm = c->tc ? ((V + 127) / 128) * 4 : 1;   // argmax partials per row (tile x lane quarter)
   c->topk_slice = (V + SM_SLOTS - 1) / SM_SLOTS;
   c->topk_blocks = (V + c->topk_slice - 1) / c->topk_slice;
   c->nsplit_attn = c->tc ? (SM_SLOTS / (f.n_heads * B) < 1 ? 1 : (SM_SLOTS / (f.n_heads * B) > 16 ? 16 : SM_SLOTS / (f.n_heads * B))) : 1;
@@ -218,11 +296,13 @@ size_t carve(spec_ctx* c, void* base) {
     for (int i = 0; i < 3; ++i) {
       size_t m = Ms[i];
       if (c->tc) {
-        int mt = mt_for_rows((int)m), mtiles = ((int)m + mt - 1) / mt;
-        size_t a = (size_t)splits_for((c->Nqkv + 127) / 128, mtiles, d) * m * c->Nqkv;
-        size_t o = (size_t)splits_for((d + 127) / 128, mtiles, HD) * m * d;
-        size_t dn = (size_t)splits_for((d + 127) / 128, mtiles, F) * m * d;
-        pf = std::max(pf, std::max(a, std::max(o, dn)));
+        int KD = f.n_kv_heads * f.head_dim;
+        int r_qkv[3] = {HD, KD, KD}, r_o[1] = {d}, r_gu[2] = {F, F}, r_dn[1] = {d};
+        GemmPlan g;
+        if (plan_gemm((int)m, d, 3, r_qkv, SM_SLOTS, false, &g)) pf = std::max(pf, plan_part_floats(g));
+        if (plan_gemm((int)m, HD, 1, r_o, SM_SLOTS, false, &g)) pf = std::max(pf, plan_part_floats(g));
+        if (plan_gemm((int)m, d, 2, r_gu, SM_SLOTS, false, &g)) pf = std::max(pf, plan_part_floats(g));
+        if (plan_gemm((int)m, F, 1, r_dn, SM_SLOTS, false, &g)) pf = std::max(pf, plan_part_floats(g));
       } else {
         pf = std::max(pf, std::max(m * (size_t)c->Nqkv, 2 * m * (size_t)F));
       }
@@ -231,7 +311,7 @@ size_t carve(spec_ctx* c, void* base) {
   c->part_floats = pf;
   c->d_part = b.take<float>(pf, 1024);
   c->d_logits = c->keep_logits ? b.take<float>((size_t)Mlog * V, 1024) : nullptr;
-  c->d_pval = b.take<float>((size_t)c->ntile_lm * M); c->d_pidx = b.take<int>((size_t)c->ntile_lm * M);
+  c->d_pval = b.take<float>((size_t)c->ntile_lm * M, 1024); c->d_pidx = b.take<int>((size_t)c->ntile_lm * M, 1024);
   c->d_part_o = c->tc ? b.take<float>((size_t)c->nsplit_attn * M * HD, 1024) : nullptr;
   c->d_part_ml = c->tc ? b.take<float>((size_t)c->nsplit_attn * M * f.n_heads * 2) : nullptr;
   c->d_pk_val = b.take<float>((size_t)c->topk_blocks * B * (K ? K : 1) * c->kmax);
@@ -289,49 +369,34 @@ Rows make_rows(spec_ctx* c, int R, bool chain) {
   return r;
 }
 
-// ---- tensor-core linear launch (bf16) ----
-template <int MT, int EPI>
-int launch_gemm_tc_mt(spec_ctx* c, cudaStream_t st, const CUtensorMap* a, const CUtensorMap* a2, const CUtensorMap* bm,
-                      const GemmTcParams& p, int n_tiles, int m_tiles, long long* launches) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc<MT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmTcCfg<MT>::SMEM_BYTES) != cudaSuccess)
-      return SPEC_E_CUDA;
-    attr_set = true;
+// ---- tensor-core linear (bf16): partial sums of x[M,K] * [mats]^T ----
+// kind: SPEC_PROFILE_* of the call site. On success *view describes the partial sums.
+int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* const* mats, const int* rows, int kind,
+             PartView* view) {
+  GemmPlan g;
+  if (!plan_gemm(M, K, n_mats, rows, c->gemm_ctas, false, &g)) return c->fail(SPEC_E_BADARG, "unsupported linear shape");
+  if (plan_part_floats(g) > c->part_floats) return c->fail(SPEC_E_NOMEM, "partial-sum scratch too small");
+  StreamTmaps tm{};
+  for (int i = 0; i < n_mats; ++i) {
+    const CUtensorMap* t = c->tmap(mats[i], rows[i], K, 128);
+    if (!t) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed (weights)");
+    tm.a[i] = *t;
   }
-  dim3 grid(n_tiles, p.splits, m_tiles);
-  gemm_tc<MT, EPI><<<grid, 128, GemmTcCfg<MT>::SMEM_BYTES, st>>>(*a, *a2, *bm, p);
-  if (launches) ++*launches;
-  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_E_CUDA;
-}
-template <int EPI>
-int launch_gemm_tc(spec_ctx* c, cudaStream_t st, int mt, const CUtensorMap* a, const CUtensorMap* a2, const CUtensorMap* bm,
-                   const GemmTcParams& p, int n_tiles, int m_tiles, long long* launches) {
-  switch (mt) {
-    case 16: return launch_gemm_tc_mt<16, EPI>(c, st, a, a2, bm, p, n_tiles, m_tiles, launches);
-    case 32: return launch_gemm_tc_mt<32, EPI>(c, st, a, a2, bm, p, n_tiles, m_tiles, launches);
-    case 64: return launch_gemm_tc_mt<64, EPI>(c, st, a, a2, bm, p, n_tiles, m_tiles, launches);
-    default: return launch_gemm_tc_mt<128, EPI>(c, st, a, a2, bm, p, n_tiles, m_tiles, launches);
-  }
-}
-
-// y partials = x[M,K] W[N,K]^T; returns the number of K slices used (>0) or a negative error.
-int linear_tc_partial(spec_ctx* c, const void* x, const void* W, int M, int N, int K, float* out, int kind) {
-  int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (N + 127) / 128;
-  int s = splits_for(n_tiles, m_tiles, K);
-  if ((size_t)s * M * N > c->part_floats && out == c->d_part) return c->fail(SPEC_E_NOMEM, "split-K scratch too small");
-  const CUtensorMap* ta = c->tmap(W, N, K, 64);
-  const CUtensorMap* tb = c->tmap(x, std::max<size_t>(round_up(M, 16), mt), K, mt);
-  if (!ta || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
-  GemmTcParams p{};
-  p.M = M; p.N = N; p.K = K; p.splits = s; p.a2_row_offset = 64; p.tile_rows = 128;
-  p.out = out; p.split_stride = (size_t)M * N; p.ldo = N; p.status = c->d_status;
+  const CUtensorMap* tb = c->tmap(x, std::max<size_t>(round_up(M, 16), g.MT), K, g.MT);
+  if (!tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed (activations)");
+  tm.b = *tb;
+  g.p.part = c->d_part;
+  g.p.slot_stride = (size_t)M * g.p.n_tiles * 128;
+  g.p.l2_prefetch = c->l2_prefetch;
+  g.p.status = c->d_status;
   {
     ProfScope ps(c, kind);
-    if (launch_gemm_tc<EPI_PARTIAL>(c, c->stream, mt, ta, ta, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
-      return c->fail(SPEC_E_CUDA, std::string("gemm_tc launch: ") + cudaGetErrorString(cudaGetLastError()));
+    cudaError_t e = launch_gs(c->stream, c->pdl, g, tm);
+    c->launches++;
+    if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_stream launch: ") + cudaGetErrorString(e));
   }
-  return s;
+  *view = plan_view(g);
+  return SPEC_OK;
 }
 
 template <typename T>
@@ -343,11 +408,108 @@ int linear_simple(spec_ctx* c, const T* x, int ldx, const T* W, float* y, int ld
   return SPEC_OK;
 }
 
-// One pass of the base model over M = B*R rows whose tokens/positions/slots are prepared
-// and whose embeddings are in d_x. lm_rows > 0: run lm_head over the first lm_rows rows of
-// `lm_src` (bf16/float operand rows) and leave per-row argmax partials.
+#define KLAUNCH(name, kernel, grid, block, smem, ...)                                            \
+  do {                                                                                         \
+    cudaError_t e_ = launch_k(c->pdl, kernel, grid, block, smem, c->stream, __VA_ARGS__);      \
+    c->launches++;                                                                             \
+    if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string(name) + ": " + cudaGetErrorString(e_)); \
+  } while (0)
+
+int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l) {
+  const spec_config& f = c->cfg;
+  int H = f.n_heads, D = f.head_dim, HD = H * D, M = c->B * R;
+  AttnTcArgs a{};
+  a.q = static_cast<const bf16*>(c->d_q); a.part_o = c->d_part_o; a.part_ml = c->d_part_ml;
+  a.pool = static_cast<const bf16*>(c->d_pool); a.g = c->geom; a.page_table = c->d_page_table; a.rows = rows;
+  a.layer = l; a.H = H; a.nsplit = c->nsplit_attn; a.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+  a.status = c->d_status;
+  dim3 grid(H, c->nsplit_attn, c->B);
+  int nw = (R + 15) / 16;
+  size_t rowb = (size_t)D * 2;
+#define ATTN_CASE(HDV, NWV)                                                                              \
+  {                                                                                                    \
+    size_t sm = (size_t)NWV * 16 * rowb + 4 * 64 * rowb + 64;                                          \
+    static bool set_ = false;                                                                          \
+    if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_tc<HDV, NWV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); set_ = true; } \
+    KLAUNCH("attention_tc", (attention_tc<HDV, NWV>), grid, dim3(NWV * 32), sm, a);                    \
+  }
+  {
+    ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
+    if (D == 128) {
+      if (nw <= 1) ATTN_CASE(128, 1) else if (nw <= 2) ATTN_CASE(128, 2) else if (nw <= 4) ATTN_CASE(128, 4) else ATTN_CASE(128, 8)
+    } else {
+      if (nw <= 1) ATTN_CASE(64, 1) else if (nw <= 2) ATTN_CASE(64, 2) else if (nw <= 4) ATTN_CASE(64, 4) else ATTN_CASE(64, 8)
+    }
+  }
+#undef ATTN_CASE
+  size_t total = (size_t)M * HD / 4;
+  KLAUNCH("attention_combine", attention_combine, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, c->d_part_o, c->d_part_ml,
+          c->nsplit_attn, rows, H, D, static_cast<bf16*>(c->d_attn));
+  return SPEC_OK;
+}
+
+// One pass of the base model over M = B*R rows whose tokens/positions/slots are prepared and
+// whose embeddings are in d_x: bf16 tensor-core path. Leaves the final hidden state in d_hid
+// (float32) and d_hq (bf16).
+int forward_layers_tc(spec_ctx* c, int R, bool chain) {
+  const spec_config& f = c->cfg;
+  Rows rows = make_rows(c, R, chain);
+  const int M = c->B * R, d = f.d_model, F = f.d_ffn, H = f.n_heads, D = f.head_dim, HD = H * D, KD = f.n_kv_heads * D;
+  bf16* u = static_cast<bf16*>(c->d_u);
+  bf16* act = static_cast<bf16*>(c->d_act);
+  const int tiles = 128;
+  const int kp0 = (HD + tiles - 1) / tiles * tiles, vp0 = kp0 + (KD + tiles - 1) / tiles * tiles;
+  const int up0 = (F + tiles - 1) / tiles * tiles;
+  PartView pend{};              // partial sums of the previous down-projection still to be added to x
+  for (int l = 0; l < f.n_layers; ++l) {
+    KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M), dim3(NORM_THREADS), 0, c->d_x, pend, c->an[l], f.rms_eps, u, (float*)nullptr, d);
+    PartView vq{};
+    {
+      const void* mats[3] = {c->wq[l], c->wk[l], c->wv[l]};
+      int rws[3] = {HD, KD, KD};
+      int r = run_gemm(c, u, M, d, 3, mats, rws, SPEC_PROFILE_QKV, &vq);
+      if (r) return r;
+    }
+    KLAUNCH("rope_store_tc", rope_store_tc, dim3(M), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope, static_cast<bf16*>(c->d_q),
+            static_cast<bf16*>(c->d_pool), c->geom, c->d_page_table, l, H);
+    int r = launch_attention_tc(c, rows, R, l);
+    if (r) return r;
+    PartView vo{};
+    {
+      const void* mats[1] = {c->wo[l]};
+      int rws[1] = {d};
+      r = run_gemm(c, c->d_attn, M, HD, 1, mats, rws, SPEC_PROFILE_WO, &vo);
+      if (r) return r;
+    }
+    KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M), dim3(NORM_THREADS), 0, c->d_x, vo, c->fn[l], f.rms_eps, u, (float*)nullptr, d);
+    PartView vg{};
+    {
+      const void* mats[2] = {c->wg[l], c->wu[l]};
+      int rws[2] = {F, F};
+      r = run_gemm(c, u, M, d, 2, mats, rws, SPEC_PROFILE_GATE_UP, &vg);
+      if (r) return r;
+    }
+    {
+      size_t total = (size_t)M * (F / 4);
+      unsigned blocks = (unsigned)std::min<size_t>((total + 255) / 256, 2048);
+      KLAUNCH("swiglu_reduce_tc", swiglu_reduce_tc, dim3(blocks), dim3(256), 0, vg, 0, up0, act, M, F);
+    }
+    {
+      const void* mats[1] = {c->wd[l]};
+      int rws[1] = {d};
+      r = run_gemm(c, act, M, F, 1, mats, rws, SPEC_PROFILE_DOWN, &pend);
+      if (r) return r;
+    }
+  }
+  KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M), dim3(NORM_THREADS), 0, c->d_x, pend, c->final_norm, f.rms_eps,
+          static_cast<bf16*>(c->d_hq), c->d_hid, d);
+  return SPEC_OK;
+}
+
+// The same pass with the plain CUDA-core kernels (float32 configurations and the bf16 debug mode).
 template <typename T>
 int forward_layers(spec_ctx* c, int R, bool chain) {
+  if (c->tc) return forward_layers_tc(c, R, chain);
   const spec_config& f = c->cfg;
   Rows rows = make_rows(c, R, chain);
   int M = c->B * R, d = f.d_model, F = f.d_ffn, H = f.n_heads, D = f.head_dim, HD = H * D;
@@ -356,95 +518,38 @@ int forward_layers(spec_ctx* c, int R, bool chain) {
   T* attn = static_cast<T*>(c->d_attn);
   T* act = static_cast<T*>(c->d_act);
   T* pool = static_cast<T*>(c->d_pool);
-  int pending = 0;              // K slices of the previous down-projection still to be added to x
-  size_t pending_stride = 0;
+  int pending = 0;              // 1: the previous down-projection output is still to be added to x
   for (int l = 0; l < f.n_layers; ++l) {
-    rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, pending, pending_stride, c->an[l], f.rms_eps, u, nullptr, d);
+    rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, pending, (size_t)M * d, c->an[l], f.rms_eps, u, nullptr, d);
     LAUNCH_CHECK("rmsnorm_rows");
-    int sq = 1;
-    if (c->tc) {
-      if (c->qkv_fused) {
-        sq = linear_tc_partial(c, u, c->wq[l], M, c->Nqkv, d, c->d_part, SPEC_PROFILE_QKV);
-        if (sq < 0) return sq;
-      } else {
-        return c->fail(SPEC_E_BADARG, "bf16 path needs wq/wk/wv contiguous per layer");
-      }
-    } else {
-      int nk = f.n_kv_heads * D, r;
-      if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wq[l]), c->d_part, c->Nqkv, M, HD, d))) return r;
-      if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wk[l]), c->d_part + HD, c->Nqkv, M, nk, d))) return r;
-      if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wv[l]), c->d_part + HD + nk, c->Nqkv, M, nk, d))) return r;
-    }
-    rope_store<T><<<M, 256, 0, c->stream>>>(c->d_part, sq, (size_t)M * c->Nqkv, rows, c->d_rope, q, pool, c->geom, c->d_page_table, l, H);
+    int nk = f.n_kv_heads * D, r;
+    if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wq[l]), c->d_part, c->Nqkv, M, HD, d))) return r;
+    if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wk[l]), c->d_part + HD, c->Nqkv, M, nk, d))) return r;
+    if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wv[l]), c->d_part + HD + nk, c->Nqkv, M, nk, d))) return r;
+    rope_store<T><<<M, 256, 0, c->stream>>>(c->d_part, 1, (size_t)M * c->Nqkv, rows, c->d_rope, q, pool, c->geom, c->d_page_table, l, H);
     LAUNCH_CHECK("rope_store");
-    if (c->tc) {
-      AttnTcArgs a{};
-      a.q = reinterpret_cast<const bf16*>(q); a.part_o = c->d_part_o; a.part_ml = c->d_part_ml;
-      a.pool = reinterpret_cast<const bf16*>(pool); a.g = c->geom; a.page_table = c->d_page_table; a.rows = rows;
-      a.layer = l; a.H = H; a.nsplit = c->nsplit_attn; a.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
-      a.status = c->d_status;
-      dim3 grid(H, c->nsplit_attn, c->B);
-      int nw = (R + 15) / 16;
-      size_t rowb = (size_t)D * 2;
-#define ATTN_CASE(HDV, NWV)                                                                              \
-      {                                                                                                  \
-        size_t sm = (size_t)NWV * 16 * rowb + 4 * 64 * rowb + 64;                                        \
-        static bool set_ = false;                                                                        \
-        if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_tc<HDV, NWV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); set_ = true; } \
-        attention_tc<HDV, NWV><<<grid, NWV * 32, sm, c->stream>>>(a);                                    \
-      }
-      ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
-      if (D == 128) {
-        if (nw <= 1) ATTN_CASE(128, 1) else if (nw <= 2) ATTN_CASE(128, 2) else if (nw <= 4) ATTN_CASE(128, 4) else ATTN_CASE(128, 8)
-      } else {
-        if (nw <= 1) ATTN_CASE(64, 1) else if (nw <= 2) ATTN_CASE(64, 2) else if (nw <= 4) ATTN_CASE(64, 4) else ATTN_CASE(64, 8)
-      }
-#undef ATTN_CASE
-      LAUNCH_CHECK("attention_tc");
-      size_t total = (size_t)M * HD / 4;
-      attention_combine<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(c->d_part_o, c->d_part_ml, c->nsplit_attn, rows, H, D,
-                                                                                reinterpret_cast<bf16*>(attn));
-      LAUNCH_CHECK("attention_combine");
-    } else {
+    {
       dim3 grid(H, c->B, (R + 3) / 4);
       attention_simple<T><<<grid, 128, 0, c->stream>>>(q, attn, pool, c->geom, c->d_page_table, rows, l, H, 1.0f / sqrtf((float)D));
       LAUNCH_CHECK("attention_simple");
     }
-    // output projection + residual + FFN norm
-    int so = 1;
-    if (c->tc) { so = linear_tc_partial(c, attn, c->wo[l], M, d, HD, c->d_part, SPEC_PROFILE_WO); if (so < 0) return so; }
-    else { int r = linear_simple<T>(c, attn, HD, static_cast<const T*>(c->wo[l]), c->d_part, d, M, d, HD); if (r) return r; }
-    rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, so, (size_t)M * d, c->fn[l], f.rms_eps, u, nullptr, d);
+    if ((r = linear_simple<T>(c, attn, HD, static_cast<const T*>(c->wo[l]), c->d_part, d, M, d, HD))) return r;
+    rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, 1, (size_t)M * d, c->fn[l], f.rms_eps, u, nullptr, d);
     LAUNCH_CHECK("rmsnorm_rows");
-    // SwiGLU FFN
-    if (c->tc) {
-      int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (F + 63) / 64;
-      const CUtensorMap* tg = c->tmap(c->wg[l], F, d, 64);
-      const CUtensorMap* tu = c->tmap(c->wu[l], F, d, 64);
-      const CUtensorMap* tb = c->tmap(u, std::max<size_t>(round_up(M, 16), mt), d, mt);
-      if (!tg || !tu || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
-      GemmTcParams p{};
-      p.M = M; p.N = F; p.K = d; p.splits = 1; p.a2_row_offset = 0; p.tile_rows = 64;
-      p.act = reinterpret_cast<bf16*>(act); p.ld_act = F; p.status = c->d_status;
-      ProfScope ps(c, SPEC_PROFILE_GATE_UP);
-      if (launch_gemm_tc<EPI_SWIGLU>(c, c->stream, mt, tg, tu, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
-        return c->fail(SPEC_E_CUDA, std::string("gemm_tc swiglu launch: ") + cudaGetErrorString(cudaGetLastError()));
-    } else {
+    {
       float* g = c->d_part;
       float* up = c->d_part + (size_t)M * F;
-      int r;
       if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wg[l]), g, F, M, F, d))) return r;
       if ((r = linear_simple<T>(c, u, d, static_cast<const T*>(c->wu[l]), up, F, M, F, d))) return r;
       size_t total = (size_t)M * F;
       swiglu_rows<T><<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(g, up, act, total);
       LAUNCH_CHECK("swiglu_rows");
     }
-    if (c->tc) { pending = linear_tc_partial(c, act, c->wd[l], M, d, F, c->d_part, SPEC_PROFILE_DOWN); if (pending < 0) return pending; }
-    else { int r = linear_simple<T>(c, act, F, static_cast<const T*>(c->wd[l]), c->d_part, d, M, d, F); if (r) return r; pending = 1; }
-    pending_stride = (size_t)M * d;
+    if ((r = linear_simple<T>(c, act, F, static_cast<const T*>(c->wd[l]), c->d_part, d, M, d, F))) return r;
+    pending = 1;
   }
   // final norm: hidden (float32) and its operand-typed copy
-  rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, pending, pending_stride, c->final_norm, f.rms_eps,
+  rmsnorm_rows<T><<<M, 256, 0, c->stream>>>(c->d_x, c->d_part, pending, (size_t)M * d, c->final_norm, f.rms_eps,
                                             static_cast<T*>(c->d_hq), c->d_hid, d);
   LAUNCH_CHECK("rmsnorm_rows");
   return SPEC_OK;
@@ -455,16 +560,21 @@ template <typename T>
 int lm_head_argmax(spec_ctx* c, const T* src, int M) {
   const spec_config& f = c->cfg;
   if (c->tc) {
-    int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = c->ntile_lm;
-    const CUtensorMap* ta = c->tmap(c->lm_head, f.vocab, f.d_model, 64);
-    const CUtensorMap* tb = c->tmap(src, std::max<size_t>(round_up(M, 16), mt), f.d_model, mt);
+    GemmPlan g;
+    int rws[1] = {f.vocab};
+    if (!plan_gemm(M, f.d_model, 1, rws, c->gemm_ctas, true, &g)) return c->fail(SPEC_E_BADARG, "unsupported lm_head shape");
+    StreamTmaps tm{};
+    const CUtensorMap* ta = c->tmap(c->lm_head, f.vocab, f.d_model, 128);
+    const CUtensorMap* tb = c->tmap(src, std::max<size_t>(round_up(M, 16), g.MT), f.d_model, g.MT);
     if (!ta || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
-    GemmTcParams p{};
-    p.M = M; p.N = f.vocab; p.K = f.d_model; p.splits = 1; p.a2_row_offset = 64; p.tile_rows = 128;
-    p.logits = c->keep_logits ? c->d_logits : nullptr; p.pval = c->d_pval; p.pidx = c->d_pidx; p.pstride = c->Mcap;
-    p.status = c->d_status;
-    if (launch_gemm_tc<EPI_ARGMAX>(c, c->stream, mt, ta, ta, tb, p, n_tiles, m_tiles, &c->launches) != SPEC_OK)
-      return c->fail(SPEC_E_CUDA, std::string("gemm_tc lm_head launch: ") + cudaGetErrorString(cudaGetLastError()));
+    tm.a[0] = *ta; tm.b = *tb;
+    g.p.logits = c->keep_logits ? c->d_logits : nullptr; g.p.ld_logits = f.vocab;
+    g.p.pval = c->d_pval; g.p.pidx = c->d_pidx;
+    g.p.l2_prefetch = c->l2_prefetch;
+    g.p.status = c->d_status;
+    cudaError_t e = launch_gs(c->stream, c->pdl, g, tm);
+    c->launches++;
+    if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_stream lm_head launch: ") + cudaGetErrorString(e));
   } else {
     int r = linear_simple<T>(c, src, f.d_model, static_cast<const T*>(c->lm_head), c->d_logits, f.vocab, M, f.vocab, f.d_model);
     if (r) return r;
@@ -477,7 +587,7 @@ int lm_head_argmax(spec_ctx* c, const T* src, int M) {
 AcceptArgs make_accept(spec_ctx* c, int R, int mode) {
   AcceptArgs a{};
   a.rows = make_rows(c, R, false);
-  a.pval = c->d_pval; a.pidx = c->d_pidx; a.ntile = c->ntile_lm; a.pstride = c->Mcap;
+  a.pval = c->d_pval; a.pidx = c->d_pidx; a.ntile = c->ntile_lm;
   a.parent = c->d_parent; a.depth = c->d_depth; a.edge_ok = nullptr;
   a.K = c->K; a.frag_token = c->cfg.frag_token; a.d = c->cfg.d_model; a.mode = mode;
   a.hid = c->d_hid; a.am = c->d_am; a.path = c->d_path; a.count = c->d_count; a.out_tok = c->d_out_tok;
@@ -533,8 +643,7 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
   int r = lm_head_argmax<T>(c, static_cast<const T*>(c->d_hq_last), batch);
   if (r) return r;
   AcceptArgs a = make_accept(c, 1, 1);
-  accept_kernel<<<batch, 128, 0, c->stream>>>(a);
-  LAUNCH_CHECK("accept_kernel");
+  KLAUNCH("accept_kernel", accept_kernel, dim3(batch), dim3(256), 0, a);
   r = check_status(c);
   if (r) return r;
   c->n_hi.assign(batch, 0);
@@ -600,8 +709,7 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     LAUNCH_CHECK("typical_edges");
     a.edge_ok = c->d_edge;
   }
-  accept_kernel<<<B, 128, 0, c->stream>>>(a);
-  LAUNCH_CHECK("accept_kernel");
+  KLAUNCH("accept_kernel", accept_kernel, dim3(B), dim3(256), 0, a);
   cudaEventRecord(c->phase_ev[4], c->stream);
   // (5) KV compaction
   dim3 gc(f.n_layers * 2 * f.n_kv_heads, B);
@@ -684,7 +792,6 @@ int spec_create(const spec_config* cfg, const spec_weights* w, const spec_tree* 
     if (static_cast<const uint8_t*>(w->wk[l]) != q0 + qn || static_cast<const uint8_t*>(w->wv[l]) != q0 + qn + kn) c->qkv_fused = false;
   }
   for (int k = 0; k < c->K; ++k) { c->mw.push_back(w->medusa_w[k]); c->mb.push_back(w->medusa_b[k]); }
-  if (c->tc && !c->qkv_fused) { g_create_error = "bf16 path needs wq/wk/wv of a layer contiguous (wq, wk, wv)"; delete c; return SPEC_E_BADARG; }
   if (c->tc && !get_encode_fn()) { g_create_error = "cuTensorMapEncodeTiled entry point unavailable"; delete c; return SPEC_E_CUDA; }
 
   // host-made tables: tree arrays, ancestor bitsets (tree and chain), page table, RoPE table
@@ -794,6 +901,20 @@ int64_t spec_query(const spec_ctx* c, int32_t what) {
   }
 }
 
+int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
+  if (!c) return SPEC_E_BADARG;
+  switch (what) {
+    case SPEC_OPT_PDL: c->pdl = value != 0; return SPEC_OK;
+    case SPEC_OPT_GEMM_CTAS:
+      if (value < 1 || value > SM_SLOTS) return c->fail(SPEC_E_BADARG, "gemm CTA count out of range");
+      c->gemm_ctas = value; return SPEC_OK;
+    case SPEC_OPT_L2_PREFETCH:
+      if (value < 0 || value > 64) return c->fail(SPEC_E_BADARG, "L2 prefetch depth out of range");
+      c->l2_prefetch = value; return SPEC_OK;
+    default: return c->fail(SPEC_E_BADARG, "unknown option");
+  }
+}
+
 int spec_last_step_phase_ms(spec_ctx* c, float* ms) {
   if (!c || !ms) return SPEC_E_BADARG;
   if (!c->phase_valid) return c->fail(SPEC_E_STATE, "no step has run");
@@ -881,9 +1002,48 @@ int spec_debug_read_kv(spec_ctx* c, int32_t seq, int32_t layer, int32_t slot0, i
   return SPEC_OK;
 }
 
+namespace {
+// Shared body of the two stand-alone linear entry points (bf16): scratch holds the partial
+// sums followed by the four-int status word.
+int op_linear_bf16(const void* x, const void* w, float* y, int M, int N, int K, int ctas, float* scratch,
+                   size_t scratch_floats, cudaStream_t st) {
+  GemmPlan g;
+  int rws[1] = {N};
+  if (!plan_gemm(M, K, 1, rws, ctas, false, &g)) return SPEC_E_BADARG;
+  StreamTmaps tm{};
+  if (!make_tmap(&tm.a[0], w, N, K, 128) || !make_tmap(&tm.b, x, M, K, g.MT)) return SPEC_E_CUDA;
+  g.p.part = scratch;
+  g.p.slot_stride = (size_t)M * g.p.n_tiles * 128;
+  g.p.l2_prefetch = 0;
+  g.p.status = reinterpret_cast<int*>(scratch + scratch_floats);
+  // the status word must start at zero; the partial sums are fully overwritten before they are read
+  if (cudaMemsetAsync(g.p.status, 0, 16, st) != cudaSuccess) return SPEC_E_CUDA;
+  if (launch_gs(st, false, g, tm) != cudaSuccess) return SPEC_E_CUDA;
+  size_t total = (size_t)M * ((N + 3) / 4);
+  part_sum_rows<<<(unsigned)std::min<size_t>((total + 255) / 256, 4096), 256, 0, st>>>(plan_view(g), y, M, N);
+  if (cudaGetLastError() != cudaSuccess) return SPEC_E_CUDA;
+  int stw[4];
+  if (cudaMemcpyAsync(stw, g.p.status, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return SPEC_E_CUDA;
+  return stw[0] == 0 ? SPEC_OK : SPEC_E_TIMEOUT;
+}
+bool op_linear_args_ok(int32_t dtype, const void* x, const void* w, const float* y, int M, int N, int K, int ctas) {
+  if (!x || !w || !y || M < 1 || N < 1 || K < 8 || K % 8 || M > 2048) return false;
+  if (dtype == 0) return true;
+  return dtype == 1 && K % 64 == 0 && M % 16 == 0 && N >= 128 && ctas >= 1 && ctas <= 1024;
+}
+}  // namespace
+
+size_t spec_op_linear_scratch_floats(int32_t M, int32_t N, int32_t K, int32_t ctas) {
+  GemmPlan g;
+  int rws[1] = {N};
+  if (M < 1 || N < 1 || ctas < 1 || !plan_gemm(M, K, 1, rws, ctas, false, &g)) return 0;
+  return plan_part_floats(g);
+}
+
 int spec_op_linear(int32_t dtype, const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                   int32_t splits, float* scratch, void* cuda_stream) {
-  if (!x || !w || !y || M < 1 || N < 1 || K < 8 || K % 8 || M > 2048) return SPEC_E_BADARG;
+                   int32_t ctas, float* scratch, void* cuda_stream) {
+  if (!op_linear_args_ok(dtype, x, w, y, M, N, K, ctas)) return SPEC_E_BADARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (dtype == 0) {
     constexpr int MC = 8;
@@ -891,32 +1051,15 @@ int spec_op_linear(int32_t dtype, const void* x, const void* w, float* y, int32_
     linear_rows<float, MC><<<grid, 256, 0, st>>>(static_cast<const float*>(x), K, static_cast<const float*>(w), y, N, M, N, K);
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_E_CUDA;
   }
-  if (dtype != 1 || K % 64 || splits < 1 || splits > K / 64 || !scratch) return SPEC_E_BADARG;
-  if (M % 16) return SPEC_E_BADARG;   // the activation map is declared over whole 16-row groups
-  int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (N + 127) / 128;
-  CUtensorMap ta, tb;
-  if (!make_tmap(&ta, w, N, K, 64) || !make_tmap(&tb, x, M, K, mt)) return SPEC_E_CUDA;
-  GemmTcParams p{};
-  p.M = M; p.N = N; p.K = K; p.splits = splits; p.a2_row_offset = 64; p.tile_rows = 128;
-  p.out = scratch; p.split_stride = (size_t)M * N; p.ldo = N;
-  // the status word of a stand-alone call lives at the end of the scratch buffer
-  p.status = reinterpret_cast<int*>(scratch + (size_t)splits * M * N);
-  if (cudaMemsetAsync(p.status, 0, 16, st) != cudaSuccess) return SPEC_E_CUDA;
-  int r = launch_gemm_tc<EPI_PARTIAL>(nullptr, st, mt, &ta, &ta, &tb, p, n_tiles, m_tiles, nullptr);
-  if (r) return r;
-  size_t total = (size_t)M * N;
-  sum_partials<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(scratch, splits, total, y);
-  if (cudaGetLastError() != cudaSuccess) return SPEC_E_CUDA;
-  int stw[4];
-  if (cudaMemcpyAsync(stw, p.status, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
-    return SPEC_E_CUDA;
-  return stw[0] == 0 ? SPEC_OK : SPEC_E_TIMEOUT;
+  if (!scratch) return SPEC_E_BADARG;
+  return op_linear_bf16(x, w, y, M, N, K, ctas, scratch, spec_op_linear_scratch_floats(M, N, K, ctas), st);
 }
 
+}  // extern "C"
 
 // ---- the linear operation for callers that cannot allocate device memory ----
-// The K-slice partial sums and the status word of spec_op_linear_static live here instead of in
-// a caller-provided buffer. Every context that loads the library holds these bytes until exit.
+// The partial sums and the status word of spec_op_linear_static live here instead of in a
+// caller-provided buffer. Every context that loads the library holds these bytes until exit.
 static __device__ __align__(256) float g_static_linear_scratch[SPEC_STATIC_SCRATCH_FLOATS + 4];
 
 namespace {
@@ -924,9 +1067,9 @@ constexpr int kMaxDevices = 64;
 float* g_static_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
 }  // namespace
 
-int spec_op_linear_static(int32_t dtype, const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                          int32_t splits, void* cuda_stream) {
-  if (!x || !w || !y || M < 1 || N < 1 || K < 8 || K % 8 || M > 2048) { g_create_error = "spec_op_linear_static: bad argument"; return SPEC_E_BADARG; }
+extern "C" int spec_op_linear_static(int32_t dtype, const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                                     int32_t ctas, void* cuda_stream) {
+  if (!op_linear_args_ok(dtype, x, w, y, M, N, K, ctas)) { g_create_error = "spec_op_linear_static: bad argument"; return SPEC_E_BADARG; }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (dtype == 0) {
     constexpr int MC = 8;
@@ -934,11 +1077,12 @@ int spec_op_linear_static(int32_t dtype, const void* x, const void* w, float* y,
     linear_rows<float, MC><<<grid, 256, 0, st>>>(static_cast<const float*>(x), K, static_cast<const float*>(w), y, N, M, N, K);
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_E_CUDA;
   }
-  if (dtype != 1 || K % 64 || splits < 1 || splits > K / 64 || M % 16) { g_create_error = "spec_op_linear_static: bad argument"; return SPEC_E_BADARG; }
-  if ((size_t)splits * M * N > (size_t)SPEC_STATIC_SCRATCH_FLOATS) {
-    char buf[160];
-    snprintf(buf, sizeof(buf), "spec_op_linear_static: splits*M*N = %zu floats exceeds the built-in scratch of %u floats",
-             (size_t)splits * M * N, (unsigned)SPEC_STATIC_SCRATCH_FLOATS);
+  const size_t need = spec_op_linear_scratch_floats(M, N, K, ctas);
+  if (need == 0) { g_create_error = "spec_op_linear_static: bad argument"; return SPEC_E_BADARG; }
+  if (need > (size_t)SPEC_STATIC_SCRATCH_FLOATS) {
+    char buf[200];
+    snprintf(buf, sizeof(buf), "spec_op_linear_static: %zu floats of partial sums exceeds the built-in scratch of %u floats",
+             need, (unsigned)SPEC_STATIC_SCRATCH_FLOATS);
     g_create_error = buf;
     return SPEC_E_NOMEM;
   }
@@ -948,31 +1092,14 @@ int spec_op_linear_static(int32_t dtype, const void* x, const void* w, float* y,
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { g_create_error = "spec_op_linear_static: cudaGetDevice failed"; return SPEC_E_CUDA; }
   float* scratch = g_static_scratch_addr[dev];
   if (!scratch) {
-    void* p = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(&p, g_static_linear_scratch);
-    if (e != cudaSuccess || !p) { g_create_error = std::string("spec_op_linear_static: cudaGetSymbolAddress: ") + cudaGetErrorString(e); return SPEC_E_CUDA; }
-    scratch = static_cast<float*>(p);
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_linear_scratch);
+    if (e != cudaSuccess || !ptr) { g_create_error = std::string("spec_op_linear_static: cudaGetSymbolAddress: ") + cudaGetErrorString(e); return SPEC_E_CUDA; }
+    scratch = static_cast<float*>(ptr);
     g_static_scratch_addr[dev] = scratch;
   }
-  int mt = mt_for_rows(M), m_tiles = (M + mt - 1) / mt, n_tiles = (N + 127) / 128;
-  CUtensorMap ta, tb;
-  if (!make_tmap(&ta, w, N, K, 64) || !make_tmap(&tb, x, M, K, mt)) { g_create_error = "spec_op_linear_static: cuTensorMapEncodeTiled failed"; return SPEC_E_CUDA; }
-  GemmTcParams p{};
-  p.M = M; p.N = N; p.K = K; p.splits = splits; p.a2_row_offset = 64; p.tile_rows = 128;
-  p.out = scratch; p.split_stride = (size_t)M * N; p.ldo = N;
-  p.status = reinterpret_cast<int*>(scratch + (size_t)SPEC_STATIC_SCRATCH_FLOATS);
-  // the array keeps the previous call's contents: the status word must start at zero (the
-  // partial sums are fully overwritten before they are read)
-  if (cudaMemsetAsync(p.status, 0, 16, st) != cudaSuccess) return SPEC_E_CUDA;
-  int r = launch_gemm_tc<EPI_PARTIAL>(nullptr, st, mt, &ta, &ta, &tb, p, n_tiles, m_tiles, nullptr);
-  if (r) return r;
-  size_t total = (size_t)M * N;
-  sum_partials<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(scratch, splits, total, y);
-  if (cudaGetLastError() != cudaSuccess) return SPEC_E_CUDA;
-  int stw[4];
-  if (cudaMemcpyAsync(stw, p.status, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
-    return SPEC_E_CUDA;
-  return stw[0] == 0 ? SPEC_OK : SPEC_E_TIMEOUT;
+  // the status word sits at the fixed end of the array
+  int r = op_linear_bf16(x, w, y, M, N, K, ctas, scratch, (size_t)SPEC_STATIC_SCRATCH_FLOATS, st);
+  if (r) g_create_error = "spec_op_linear_static: launch or device status failed";
+  return r;
 }
-
-}  // extern "C"

@@ -129,9 +129,10 @@ def test_typical_acceptance_mode(torch):
     assert rep.steps > 0
 
 
-@pytest.mark.parametrize("M,N,K,splits", [(16, 128, 64, 1), (64, 384, 256, 2), (64, 4096, 4096, 3),
-                                          (128, 1000, 704, 2), (32, 200, 128, 1), (256, 512, 512, 4)])
-def test_op_linear_bf16_vs_oracle_matmul(torch, M, N, K, splits):
+@pytest.mark.parametrize("M,N,K,ctas", [(16, 128, 64, 1), (64, 384, 256, 2), (64, 4096, 4096, 296),
+                                        (128, 1000, 704, 7), (32, 200, 128, 3), (256, 512, 512, 148),
+                                        (64, 12288, 4096, 296), (48, 1000, 1408, 37)])
+def test_op_linear_bf16_vs_oracle_matmul(torch, M, N, K, ctas):
     from oracle.numerics import round_bf16
     from paper_2503_14153_b200 import spec_op_linear
     rng = np.random.default_rng(M * 7 + N)
@@ -139,7 +140,7 @@ def test_op_linear_bf16_vs_oracle_matmul(torch, M, N, K, splits):
     w = round_bf16((rng.standard_normal((N, K)) * 0.05).astype(np.float32))
     ref = x @ w.T
     y = spec_op_linear(torch.from_numpy(x.astype(np.float32)).cuda().to(torch.bfloat16),
-                       torch.from_numpy(w.astype(np.float32)).cuda().to(torch.bfloat16), splits).cpu().numpy()
+                       torch.from_numpy(w.astype(np.float32)).cuda().to(torch.bfloat16), ctas).cpu().numpy()
     err = np.abs(y - ref).max() / np.abs(ref).max()
     assert err < 1e-5, err
 

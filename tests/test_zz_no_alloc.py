@@ -37,16 +37,16 @@ def test_static_scratch_linear_matches_caller_scratch_linear_twice(torch):
     from paper_2503_14153_b200 import spec_op_linear, spec_op_linear_static
     # two different problems back to back: the second starts with the first's leftovers in the scratch
     cases = [(64, 1000, 704, 3, 11), (32, 384, 256, 2, 12)]
-    for M, N, K, splits, seed in cases:
+    for M, N, K, ctas, seed in cases:
         x, w = _operands(torch, M, N, K, seed, torch.bfloat16)
-        want = spec_op_linear(x, w, splits)
+        want = spec_op_linear(x, w, ctas)
         y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")   # caller-owned output
         before = torch.cuda.memory_stats()["allocation.all.allocated"]    # cumulative count of allocations
-        got = spec_op_linear_static(x, w, y, splits)
+        got = spec_op_linear_static(x, w, y, ctas)
         assert torch.cuda.memory_stats()["allocation.all.allocated"] == before   # none came from torch's allocator
         torch.cuda.synchronize()
         err = (got - want).abs().max().item() / want.abs().max().item()
-        assert err <= TOL, (M, N, K, splits, err)
+        assert err <= TOL, (M, N, K, ctas, err)
     # the same problem again: identical bits both times
     x, w = _operands(torch, 64, 1000, 704, 11, torch.bfloat16)
     y1 = spec_op_linear_static(x, w, torch.empty((64, 1000), dtype=torch.float32, device="cuda"), 3).clone()
@@ -65,10 +65,11 @@ def test_static_scratch_linear_float32(torch):
 def test_static_scratch_linear_refuses_oversize(torch):
     from paper_2503_14153_b200 import SpecError, spec_op_linear_static
     from paper_2503_14153_b200.binding import STATIC_SCRATCH_FLOATS
-    M, N, K, splits = 64, 16384, 256, 4
-    assert splits * M * N > STATIC_SCRATCH_FLOATS
+    M, N, K, ctas = 64, 32768, 256, 4
+    from paper_2503_14153_b200 import load_library
+    assert load_library().spec_op_linear_scratch_floats(M, N, K, ctas) > STATIC_SCRATCH_FLOATS
     x, w = _operands(torch, M, N, K, 14, torch.bfloat16)
     y = torch.empty((M, N), dtype=torch.float32, device="cuda")
     with pytest.raises(SpecError) as ei:
-        spec_op_linear_static(x, w, y, splits)
+        spec_op_linear_static(x, w, y, ctas)
     assert ei.value.code == -3 and "exceeds the built-in scratch" in str(ei.value)
