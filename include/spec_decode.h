@@ -144,12 +144,22 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
 /* Tuning knobs of a context (defaults in brackets). SPEC_OPT_PDL [1]: launch the kernels of
  * a step with programmatic dependent launch, so that each kernel's set-up and weight prefetch
  * overlap the tail of the one before. SPEC_OPT_GEMM_CTAS [296]: persistent CTAs the
- * weight-streaming GEMM deals its work to (1..296). SPEC_OPT_L2_PREFETCH [8]: 16 KiB weight
+ * weight-streaming GEMM deals its work to (1..296). SPEC_OPT_L2_PREFETCH [0]: 16 KiB weight
  * chunks each GEMM CTA requests into L2, beyond its shared-memory ring, before it waits for the
  * previous kernel (0..64). Results do not depend on SPEC_OPT_PDL or SPEC_OPT_L2_PREFETCH;
- * SPEC_OPT_GEMM_CTAS changes the order in which partial sums are added. */
-enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2 };
+ * SPEC_OPT_GEMM_CTAS changes the order in which partial sums are added. SPEC_OPT_TRACE [0]:
+ * record a device timeline of every step (see spec_trace_read). */
+enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2, SPEC_OPT_TRACE = 3 };
 int spec_set_option(spec_ctx *ctx, int32_t what, int32_t value);
+
+/* Device timeline of the LAST step, recorded while SPEC_OPT_TRACE is on: one record per kernel
+ * launch of the step, in launch order. names: HOST [max_records][SPEC_TRACE_NAME_LEN] chars;
+ * stamps: HOST [max_records][4] nanoseconds of the GPU's global timer: earliest block start,
+ * latest block end, and for the weight-streaming GEMM the moment its first operands had landed
+ * in shared memory and the moment its last MMA was issued (all-ones / 0 when a kernel has no
+ * such mark). *n_records receives the number of launches of the step. Synchronises. */
+#define SPEC_TRACE_NAME_LEN 32
+int spec_trace_read(spec_ctx *ctx, int32_t max_records, char *names, uint64_t *stamps, int32_t *n_records);
 
 /* Device time of the five parts of the LAST step, in milliseconds, from events recorded on
  * the stream at the part boundaries: ms[0] heads + lm_head + top-k, ms[1] tree expansion and

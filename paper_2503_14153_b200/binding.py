@@ -19,13 +19,14 @@ FLAG_SIMPLE_KERNELS = 2
 PROFILE_OFF, PROFILE_GATE_UP, PROFILE_QKV, PROFILE_WO, PROFILE_DOWN, PROFILE_ATTENTION = range(6)
 
 Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB = 0, 1, 2, 3, 4
-OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH = 0, 1, 2
+OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH, OPT_TRACE = 0, 1, 2, 3
+TRACE_NAME_LEN = 32
 (DBG_TOK, DBG_POS, DBG_LOGITS, DBG_HIDDEN, DBG_ARGMAX, DBG_PATH, DBG_CAND, DBG_SEQLEN, DBG_NEXT_ROOT,
  DBG_H_LAST, DBG_STATUS) = range(11)
 
 EXPORTS = ["spec_workspace_bytes", "spec_create", "spec_prefill", "spec_step", "spec_read_generated",
            "spec_destroy", "spec_last_error", "spec_query", "spec_debug_read", "spec_debug_read_kv",
-           "spec_op_linear", "spec_op_linear_scratch_floats", "spec_op_linear_static", "spec_set_option", "spec_last_step_phase_ms", "spec_profile_kernel",
+           "spec_op_linear", "spec_op_linear_scratch_floats", "spec_op_linear_static", "spec_set_option", "spec_trace_read", "spec_last_step_phase_ms", "spec_profile_kernel",
            "spec_profile_read"]
 
 
@@ -96,6 +97,8 @@ def load_library():
     lib.spec_op_linear_scratch_floats.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32]
     lib.spec_set_option.restype = C.c_int
     lib.spec_set_option.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+    lib.spec_trace_read.restype = C.c_int
+    lib.spec_trace_read.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
     lib.spec_op_linear_static.restype = C.c_int
     lib.spec_op_linear_static.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_void_p]
@@ -263,6 +266,18 @@ class SpecDecoder:
         ms, n = C.c_double(0.0), C.c_int64(0)
         self._check(self.lib.spec_profile_read(self._ctx, C.byref(ms), C.byref(n)))
         return ms.value, n.value
+
+    def trace(self, max_records: int = 1024):
+        """Timeline of the last step (OPT_TRACE must be on): list of (name, start, end, mark_a, mark_b) in ns."""
+        names = C.create_string_buffer(max_records * TRACE_NAME_LEN)
+        stamps = np.zeros((max_records, 4), dtype=np.uint64)
+        n = C.c_int32(0)
+        self._check(self.lib.spec_trace_read(self._ctx, max_records, names, stamps.ctypes.data, C.byref(n)))
+        out = []
+        for i in range(min(n.value, max_records)):
+            nm = names.raw[i * TRACE_NAME_LEN:(i + 1) * TRACE_NAME_LEN].split(b"\0")[0].decode()
+            out.append((nm,) + tuple(int(v) for v in stamps[i]))
+        return out
 
     def set_option(self, what: int, value: int):
         self._check(self.lib.spec_set_option(self._ctx, what, value))

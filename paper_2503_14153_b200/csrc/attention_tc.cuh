@@ -47,7 +47,8 @@ struct AttnTcArgs {
 
 template <int HD, int NW>
 __global__ void __launch_bounds__(NW * 32)
-attention_tc(const AttnTcArgs a) {
+attention_tc(const AttnTcArgs a, unsigned long long* tr) {
+  KTrace kt(tr);
   constexpr int KT = 64;                      // keys per tile
   constexpr int ROWB = HD * 2;                // bytes per row
   constexpr int TILE_BYTES = KT * ROWB;
@@ -236,9 +237,11 @@ attention_tc(const AttnTcArgs a) {
 // Merges the KV splits: out[m][h*HD + d] = bf16( sum_s w_s O_s / sum_s w_s l_s ),
 // w_s = 2^(m_s - max_s m_s). One thread per (row, head, 4 dims).
 __global__ void attention_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml, int nsplit,
-                                  Rows rows, int H, int HD, bf16* __restrict__ out) {
+                                  Rows rows, int H, int HD, bf16* __restrict__ out, unsigned long long* tr) {
+  KTrace kt(tr);
   pdl_launch_dependents();
   pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   int M = rows.B * rows.R;
   size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   size_t per_row = (size_t)H * HD / 4;

@@ -76,6 +76,15 @@ struct KVGeom {
   }
 };
 
+// Per-pass row bookkeeping. Row m = b * R + i belongs to sequence b; it is valid iff
+// i < cnt[b]. n[b] cached positions precede the pass's rows of sequence b.
+struct Rows {
+  int R, B;
+  int *tok, *pos, *slot;  // [B*R]
+  int *n, *cnt;           // [B]
+  const uint32_t* anc;    // [R][4] ancestor bitsets (bit u of anc[i]: row i sees row u)
+};
+
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -203,5 +212,24 @@ __device__ __host__ __forceinline__ uint32_t make_idesc_bf16(int M, int N) {
 // programmatic dependent launch
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Optional per-launch timeline: t[0] = earliest block start, t[1] = latest block end,
+// t[2] / t[3] = kernel-specific marks (earliest / latest), all in globaltimer nanoseconds.
+// The host presets t[0] and t[2] to all-ones and t[1], t[3] to zero. t == nullptr: off.
+struct KTrace {
+  unsigned long long* t;
+  __device__ __forceinline__ explicit KTrace(unsigned long long* p) : t(p) {
+    if (t && threadIdx.x == 0) atomicMin(t, (unsigned long long)global_timer_ns());
+  }
+  __device__ __forceinline__ ~KTrace() {
+    if (t && threadIdx.x == 0) atomicMax(t + 1, (unsigned long long)global_timer_ns());
+  }
+};
+__device__ __forceinline__ void trace_mark_min(unsigned long long* t, int i) {
+  if (t) atomicMin(t + i, (unsigned long long)global_timer_ns());
+}
+__device__ __forceinline__ void trace_mark_max(unsigned long long* t, int i) {
+  if (t) atomicMax(t + i, (unsigned long long)global_timer_ns());
+}
 
 }  // namespace spec

@@ -32,7 +32,8 @@ struct SegMap {
   int total;       // n_tiles * m_tiles * KC
   __host__ __device__ __forceinline__ int lo(int c) const { return (int)(((long long)c * total) / G); }
   // CTA whose run contains unit u
-  __host__ __device__ __forceinline__ int owner(int u) const { return (int)((((long long)u + 1) * G - 1) / total); }
+  // (u + 1) * G stays below 2^31 for every unit (the host checks it), so 32-bit division serves
+  __host__ __device__ __forceinline__ int owner(int u) const { return (int)((((unsigned)u + 1u) * (unsigned)G - 1u) / (unsigned)total); }
   // number of CTAs that contribute to tile t = nt * m_tiles + mt
   __host__ __device__ __forceinline__ int nseg(int t) const { return owner((t + 1) * KC - 1) - owner(t * KC) + 1; }
 };
@@ -56,6 +57,7 @@ struct StreamGemmParams {
   float* pval;
   int* pidx;
   int* status;
+  unsigned long long* trace;        // optional timeline slot (see KTrace); [2] first operands landed, [3] last MMA issued
 };
 
 struct StreamTmaps {
@@ -63,12 +65,13 @@ struct StreamTmaps {
   CUtensorMap b;
 };
 
-template <int MT> struct StreamCfg {
+// DEEP = 0: a ring sized so that two CTAs share an SM; DEEP = 1: twice the stages, one CTA per SM.
+template <int MT, int DEEP> struct StreamCfg {
   static constexpr int BK = 64;
   static constexpr int A_BYTES = 128 * BK * 2;
   static constexpr int B_BYTES = MT * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (MT <= 32) ? 5 : (MT == 64 ? 4 : 3);
+  static constexpr int STAGES = ((MT <= 32) ? 5 : (MT == 64 ? 4 : 3)) * (DEEP ? 2 : 1);
   static constexpr int TMEM_COLS = (2 * MT < 32) ? 32 : 2 * MT;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
@@ -95,10 +98,10 @@ __device__ __forceinline__ GsUnit gs_decode(const StreamGemmParams& p, int u) {
   return w;
 }
 
-template <int MT>
-__global__ void __launch_bounds__(192, 2)
+template <int MT, int DEEP>
+__global__ void __launch_bounds__(192, DEEP ? 1 : 2)
 gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
-  using Cfg = StreamCfg<MT>;
+  using Cfg = StreamCfg<MT, DEEP>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -110,6 +113,7 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
   uint64_t* acc_empty = bars + 2 * STAGES + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
 
+  KTrace kt(p.trace);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x;
   const int KC = p.seg.KC;
@@ -199,6 +203,7 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
           const int st = done % STAGES;
           const uint32_t ph = (done / STAGES) & 1;
           if (!mbar_wait(&full[st], ph, p.status, 11)) { ok = false; break; }
+          if (v == lo) trace_mark_min(p.trace, 2);
           tc_fence_after();
           const uint32_t a_addr = smem_u32(tiles + st * Cfg::STAGE_BYTES);
           const uint64_t adesc = make_kmajor_sw128_desc(a_addr);
@@ -213,6 +218,7 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
         ++seg_i;
         u = u_end;
       }
+      trace_mark_max(p.trace, 3);
     }
   } else {
     // ---- epilogue: warps 2..5; warp w may touch tensor-memory lanes [32 (w % 4), +32) ----

@@ -17,15 +17,15 @@ struct PartView {
   const float* part;
   size_t slot_stride;
   int ld;
-  SegMap seg;
-  int MT;
+  SegMap seg;                  // how the GEMM dealt its units: gives the slots of a tile
+  int mt_shift;                // log2 of the activation rows per tile
 };
 
-constexpr int PV_UNROLL = 8;
+constexpr int PV_UNROLL = 12;
 
 // Sum over the slots of the tile that holds padded columns [colp, colp+4) of row m.
 __device__ __forceinline__ float4 part_sum4(const PartView& pv, int m, int colp) {
-  const int ns = pv.seg.nseg((colp >> 7) * pv.seg.m_tiles + m / pv.MT);
+  const int ns = pv.seg.nseg((colp >> 7) * pv.seg.m_tiles + (m >> pv.mt_shift));
   const float* src = pv.part + (size_t)m * pv.ld + colp;
   float4 v[PV_UNROLL];
 #pragma unroll
@@ -52,18 +52,29 @@ __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) 
 
 // ------------------------------------------------------------------ residual + RMSNorm
 // x[m] += sum of the partial slots (when pv.part != nullptr); u[m] = bf16(x / rms(x) * g);
-// optionally the unrounded normed row goes to hid. One CTA per row; d % 4 == 0.
-constexpr int NORM_THREADS = 512;
-constexpr int NORM_CACHE = 4;   // float4 values a thread keeps between the two passes
+// optionally the unrounded normed row goes to hid. One CTA per row; every thread issues all
+// its loads at once (one trip to L2) and keeps its values in registers for the second pass;
+// the gains do not depend on the previous kernel and are fetched before the dependency wait.
+// d % 4 == 0.
+constexpr int NORM_THREADS = 1024;
+constexpr int NORM_CACHE = 2;   // float4 values a thread keeps between the two passes
 
 __global__ void __launch_bounds__(NORM_THREADS)
 norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict__ gain, float eps,
-               bf16* __restrict__ u, float* __restrict__ hid, int d) {
+               bf16* __restrict__ u, float* __restrict__ hid, int d, unsigned long long* tr) {
+  KTrace kt(tr);
   pdl_launch_dependents();
-  pdl_wait();
   const int m = blockIdx.x;
   float* xr = x + (size_t)m * d;
   const int n4 = d >> 2;
+  float4 gk[NORM_CACHE];
+#pragma unroll
+  for (int k = 0; k < NORM_CACHE; ++k) {
+    const int c4 = threadIdx.x + k * NORM_THREADS;
+    gk[k] = c4 < n4 ? *reinterpret_cast<const float4*>(gain + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   float4 keep[NORM_CACHE];
   float ss = 0.f;
 #pragma unroll
@@ -72,7 +83,7 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
     if (c4 < n4) {
       float4 v = *reinterpret_cast<const float4*>(xr + c4 * 4);
       if (pv.part) {
-        float4 a = part_sum4(pv, m, c4 * 4);
+        const float4 a = part_sum4(pv, m, c4 * 4);
         v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
         *reinterpret_cast<float4*>(xr + c4 * 4) = v;
       }
@@ -83,7 +94,7 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
   for (int c4 = threadIdx.x + NORM_CACHE * NORM_THREADS; c4 < n4; c4 += NORM_THREADS) {
     float4 v = *reinterpret_cast<const float4*>(xr + c4 * 4);
     if (pv.part) {
-      float4 a = part_sum4(pv, m, c4 * 4);
+      const float4 a = part_sum4(pv, m, c4 * 4);
       v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
       *reinterpret_cast<float4*>(xr + c4 * 4) = v;
     }
@@ -93,70 +104,73 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
   ss = warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = threadIdx.x < (NORM_THREADS >> 5) ? red[threadIdx.x] : 0.f;
-    v = warp_sum(v);
-    if (threadIdx.x == 0) red[0] = v;
-  }
-  __syncthreads();
-  const float inv = rsqrtf(red[0] / (float)d + eps);
-  auto emit = [&](int c4, float4 v) {
-    float4 g = *reinterpret_cast<const float4*>(gain + c4 * 4);
-    float4 o = make_float4(v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < (NORM_THREADS >> 5); ++w) tot += red[w];   // same order in every thread
+  const float inv = rsqrtf(tot / (float)d + eps);
+  auto emit = [&](int c4, const float4& v, const float4& g) {
+    const float4 o = make_float4(v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
     *reinterpret_cast<uint2*>(u + (size_t)m * d + c4 * 4) = pack4_bf16(o.x, o.y, o.z, o.w);
     if (hid) *reinterpret_cast<float4*>(hid + (size_t)m * d + c4 * 4) = o;
   };
 #pragma unroll
   for (int k = 0; k < NORM_CACHE; ++k) {
     const int c4 = threadIdx.x + k * NORM_THREADS;
-    if (c4 < n4) emit(c4, keep[k]);
+    if (c4 < n4) emit(c4, keep[k], gk[k]);
   }
   for (int c4 = threadIdx.x + NORM_CACHE * NORM_THREADS; c4 < n4; c4 += NORM_THREADS)
-    emit(c4, *reinterpret_cast<const float4*>(xr + c4 * 4));
+    emit(c4, *reinterpret_cast<const float4*>(xr + c4 * 4), *reinterpret_cast<const float4*>(gain + c4 * 4));
 }
 
 // ------------------------------------------------------------------ RoPE + cache store
 // Sums the QKV partial slots, rotates q and k (rotate-half pairs (e, e + D/2), table
 // cs[pos][e] = (cos, sin)), writes q as bf16 [M][H*D] and k, v as bf16 into the paged cache at
 // the row's slot. qp0 / kp0 / vp0: first padded column of the q / k / v matrix in the partials.
-// One CTA per row; D % 8 == 0.
+// gridDim.y CTAs share a row; D % 8 == 0.
 __global__ void __launch_bounds__(256)
 rope_store_tc(const PartView pv, int qp0, int kp0, int vp0, Rows rows, const float2* __restrict__ cs,
               bf16* __restrict__ q, bf16* __restrict__ pool, KVGeom g, const int* __restrict__ page_table,
-              int layer, int H) {
+              int layer, int H, unsigned long long* tr) {
+  KTrace kt(tr);
   pdl_launch_dependents();
   pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   const int m = blockIdx.x, b = m / rows.R, i = m % rows.R;
-  if (i >= rows.cnt[b]) return;
   const int D = g.head_dim, half = D >> 1, Hkv = g.n_kv_heads;
-  const int pos = rows.pos[m], slot = rows.slot[m];
-  const int page = page_table[b * g.pages_per_seq + slot / g.page_size], prow = slot % g.page_size;
   const int q4 = half >> 2;                       // float4 groups per half head
-  const int n_rot = (H + Hkv) * q4;
-  for (int it = threadIdx.x; it < n_rot; it += blockDim.x) {
-    const int head = it / q4, e = (it % q4) * 4;
-    const int colp = (head < H ? qp0 + head * D : kp0 + (head - H) * D) + e;
-    const float4 a = part_sum4(pv, m, colp), c = part_sum4(pv, m, colp + half);
-    const float4 t01 = *reinterpret_cast<const float4*>(cs + (size_t)pos * half + e);
-    const float4 t23 = *reinterpret_cast<const float4*>(cs + (size_t)pos * half + e + 2);
-    const float r0[4] = {a.x * t01.x - c.x * t01.y, a.y * t01.z - c.y * t01.w, a.z * t23.x - c.z * t23.y, a.w * t23.z - c.w * t23.w};
-    const float r1[4] = {c.x * t01.x + a.x * t01.y, c.y * t01.z + a.y * t01.w, c.z * t23.x + a.z * t23.y, c.w * t23.z + a.w * t23.w};
-    if (head < H) {
-      bf16* dst = q + (size_t)m * H * D + head * D + e;
-      *reinterpret_cast<uint2*>(dst) = pack4_bf16(r0[0], r0[1], r0[2], r0[3]);
-      *reinterpret_cast<uint2*>(dst + half) = pack4_bf16(r1[0], r1[1], r1[2], r1[3]);
+  const int n_rot = (H + Hkv) * q4, n_v = Hkv * (D >> 2);
+  const int tid = blockIdx.y * blockDim.x + threadIdx.x, nthr = gridDim.y * blockDim.x;
+  // row bookkeeping and partial sums are independent loads: issue them together
+  const int cnt = rows.cnt[b], pos = rows.pos[m], slot = rows.slot[m];
+  for (int it = tid; it < n_rot + n_v; it += nthr) {
+    if (it < n_rot) {
+      const int head = it / q4, e = (it % q4) * 4;
+      const int colp = (head < H ? qp0 + head * D : kp0 + (head - H) * D) + e;
+      const float4 a = part_sum4(pv, m, colp), c = part_sum4(pv, m, colp + half);
+      if (i >= cnt) continue;
+      const float4 t01 = *reinterpret_cast<const float4*>(cs + (size_t)pos * half + e);
+      const float4 t23 = *reinterpret_cast<const float4*>(cs + (size_t)pos * half + e + 2);
+      const uint2 lo = pack4_bf16(a.x * t01.x - c.x * t01.y, a.y * t01.z - c.y * t01.w, a.z * t23.x - c.z * t23.y, a.w * t23.z - c.w * t23.w);
+      const uint2 hi = pack4_bf16(c.x * t01.x + a.x * t01.y, c.y * t01.z + a.y * t01.w, c.z * t23.x + a.z * t23.y, c.w * t23.z + a.w * t23.w);
+      if (head < H) {
+        bf16* dst = q + (size_t)m * H * D + head * D + e;
+        *reinterpret_cast<uint2*>(dst) = lo;
+        *reinterpret_cast<uint2*>(dst + half) = hi;
+      } else {
+        const int page = page_table[b * g.pages_per_seq + slot / g.page_size], prow = slot % g.page_size;
+        bf16* dst = pool + g.block_offset(page, layer, 0, head - H) + (size_t)prow * D;
+        *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e)) = lo;
+        *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e + half)) = hi;
+      }
     } else {
-      bf16* dst = pool + g.block_offset(page, layer, 0, head - H) + (size_t)prow * D;
-      *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e)) = pack4_bf16(r0[0], r0[1], r0[2], r0[3]);
-      *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e + half)) = pack4_bf16(r1[0], r1[1], r1[2], r1[3]);
+      const int iv = it - n_rot;
+      const int kh = iv / (D >> 2), e = (iv % (D >> 2)) * 4;
+      const float4 a = part_sum4(pv, m, vp0 + kh * D + e);
+      if (i >= cnt) continue;
+      const int page = page_table[b * g.pages_per_seq + slot / g.page_size], prow = slot % g.page_size;
+      bf16* dst = pool + g.block_offset(page, layer, 1, kh) + (size_t)prow * D;
+      *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e)) = pack4_bf16(a.x, a.y, a.z, a.w);
     }
-  }
-  const int v4 = D >> 2;
-  for (int it = threadIdx.x; it < Hkv * v4; it += blockDim.x) {
-    const int kh = it / v4, e = (it % v4) * 4;
-    const float4 a = part_sum4(pv, m, vp0 + kh * D + e);
-    bf16* dst = pool + g.block_offset(page, layer, 1, kh) + (size_t)prow * D;
-    *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e)) = pack4_bf16(a.x, a.y, a.z, a.w);
   }
 }
 
@@ -164,9 +178,11 @@ rope_store_tc(const PartView pv, int qp0, int kp0, int vp0, Rows rows, const flo
 // act[m][f] = bf16(SiLU(gate) * up), gate / up = sums of the partial slots of the gate and up
 // matrices (padded columns gp0 + f and up0 + f). F % 4 == 0.
 __global__ void __launch_bounds__(256)
-swiglu_reduce_tc(const PartView pv, int gp0, int up0, bf16* __restrict__ act, int M, int F) {
+swiglu_reduce_tc(const PartView pv, int gp0, int up0, bf16* __restrict__ act, int M, int F, unsigned long long* tr) {
+  KTrace kt(tr);
   pdl_launch_dependents();
   pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   const int f4 = F >> 2;
   const size_t total = (size_t)M * f4;
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {

@@ -8,15 +8,6 @@
 
 namespace spec {
 
-// Per-pass row bookkeeping. Row m = b * R + i belongs to sequence b; it is valid iff
-// i < cnt[b]. n[b] cached positions precede the pass's rows of sequence b.
-struct Rows {
-  int R, B;
-  int *tok, *pos, *slot;  // [B*R]
-  int *n, *cnt;           // [B]
-  const uint32_t* anc;    // [R][4] ancestor bitsets (bit u of anc[i]: row i sees row u)
-};
-
 // ------------------------------------------------------------------ row preparation
 // Verify pass: tree node i of sequence b carries candidate rank[i] of head depth[i]
 // (head 0 = the base model's own next token) and sits at position n[b] + depth[i].
@@ -24,7 +15,11 @@ template <typename T>
 __global__ void prepare_verify_rows(Rows rows, const int* __restrict__ cand, int cand_stride_b, int kmax,
                                     const int* __restrict__ depth, const int* __restrict__ rank, int capacity,
                                     const T* __restrict__ embed, float* __restrict__ x, int d, int vocab,
-                                    int* status) {
+                                    int* status, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   int m = blockIdx.x, b = m / rows.R, i = m % rows.R;
   int n = rows.n[b];
   bool ok = (n + rows.R <= capacity);
@@ -383,9 +378,11 @@ struct AcceptArgs {
 // token is the argmax at the parent, or its Eq. 1 flag is set), takes the deepest accepted node
 // (lowest index on ties), applies the fragment-integrity rule, and publishes the step's result
 // and the next step's state.
-__global__ void __launch_bounds__(256) accept_kernel(AcceptArgs a) {
+__global__ void __launch_bounds__(256) accept_kernel(AcceptArgs a, unsigned long long* tr) {
+  KTrace kt(tr);
   pdl_launch_dependents();
   pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   const int b = blockIdx.x, R = a.rows.R;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
   __shared__ int am_s[SPEC_MAX_NODES], tok_s[SPEC_MAX_NODES], par_s[SPEC_MAX_NODES], dep_s[SPEC_MAX_NODES];
@@ -478,7 +475,11 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptArgs a) {
 template <typename T>
 __global__ void compact_kv(T* __restrict__ pool, KVGeom g, const int* __restrict__ page_table,
                            const int* __restrict__ path, const int* __restrict__ count,
-                           const int* __restrict__ n_old, int K) {
+                           const int* __restrict__ n_old, int K, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   int b = blockIdx.y;
   int blk = blockIdx.x;              // (layer*2 + kv) * Hkv + head
   int head = blk % g.n_kv_heads, lk = blk / g.n_kv_heads;
@@ -501,7 +502,12 @@ __global__ void compact_kv(T* __restrict__ pool, KVGeom g, const int* __restrict
 // head k; MC sequences at a time.
 template <typename T, int MC>
 __global__ void medusa_resblock(const float* __restrict__ h_last, const T* const* __restrict__ Wk,
-                                const T* const* __restrict__ bk, T* __restrict__ r, int B, int K, int d) {
+                                const T* const* __restrict__ bk, T* __restrict__ r, int B, int K, int d,
+                                unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   constexpr int VN = Vec16<T>::N;
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int row = blockIdx.x * (blockDim.x >> 5) + warp;   // k * d + i
@@ -539,7 +545,12 @@ __global__ void medusa_resblock(const float* __restrict__ h_last, const T* const
 // the slice go to the partial lists pk_val/pk_idx [block][rows][kmax].
 template <typename T, int MC>
 __global__ void medusa_lmhead_topk(const T* __restrict__ r, const T* __restrict__ Wlm, int rows_total, int V, int d,
-                                   int slice, int kmax, float* __restrict__ pk_val, int* __restrict__ pk_idx) {
+                                   int slice, int kmax, float* __restrict__ pk_val, int* __restrict__ pk_idx,
+                                   unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   constexpr int VN = Vec16<T>::N;
   extern __shared__ float zs[];   // [MC][slice]
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
@@ -591,7 +602,11 @@ __global__ void medusa_lmhead_topk(const T* __restrict__ r, const T* __restrict_
 // the optional override table; block 0 of each sequence also writes cand[b][0][0] = root.
 __global__ void topk_merge(const float* __restrict__ pk_val, const int* __restrict__ pk_idx, int nblocks,
                            int rows_total, int K, int kmax, const int* __restrict__ root_tok,
-                           const int* __restrict__ cand_override, int* __restrict__ cand) {
+                           const int* __restrict__ cand_override, int* __restrict__ cand, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
   extern __shared__ float ms[];     // values [nblocks*kmax] then indices
   int row = blockIdx.x, b = row / K, k = row % K;
   int total = nblocks * kmax;

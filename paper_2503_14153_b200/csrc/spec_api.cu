@@ -29,6 +29,7 @@ namespace {
 thread_local std::string g_create_error = "no error";
 
 constexpr int PREFILL_ROWS = 128;   // rows per sequence in one prefill pass
+constexpr int TRACE_CAP = 1024;     // launches of one step the timeline can hold
 constexpr int SM_SLOTS = 296;       // 148 SMs x 2 co-resident GEMM CTAs
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -121,7 +122,7 @@ bool plan_gemm(int M, int K, int n_mats, const int* rows, int g_max, bool tile_g
   p.seg.KC = K / 64;
   p.seg.m_tiles = (M + g.MT - 1) / g.MT;
   long long total = (long long)tiles * p.seg.m_tiles * p.seg.KC;
-  if (total > 0x3fffffff) return false;
+  if (total > 0x3fffffff || (total + 1) * (long long)g_max >= 0x7fffffffLL) return false;
   p.seg.total = (int)total;
   p.tile_granular = tile_granular ? 1 : 0;
   long long cap = tile_granular ? (long long)tiles * p.seg.m_tiles : total;
@@ -138,28 +139,32 @@ int plan_slot_bound(const GemmPlan& g) {
 
 size_t plan_part_floats(const GemmPlan& g) { return (size_t)plan_slot_bound(g) * g.p.M * g.p.n_tiles * 128; }
 
-template <int MT>
+template <int MT, int DEEP>
 cudaError_t launch_gs_mt(cudaStream_t st, bool pdl, int grid, const StreamTmaps& tm, const StreamGemmParams& p) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_stream<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamCfg<MT>::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(gemm_stream<MT, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamCfg<MT, DEEP>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  return launch_k(pdl, gemm_stream<MT>, dim3(grid), dim3(192), (size_t)StreamCfg<MT>::SMEM_BYTES, st, tm, p);
+  return launch_k(pdl, gemm_stream<MT, DEEP>, dim3(grid), dim3(192), (size_t)StreamCfg<MT, DEEP>::SMEM_BYTES, st, tm, p);
 }
+// Grids of at most one CTA per SM get the deep ring (one resident CTA must keep the SM's share
+// of the memory pipe full by itself).
 cudaError_t launch_gs(cudaStream_t st, bool pdl, const GemmPlan& g, const StreamTmaps& tm) {
+  const bool deep = g.grid <= SM_SLOTS / 2;
   switch (g.MT) {
-    case 16: return launch_gs_mt<16>(st, pdl, g.grid, tm, g.p);
-    case 32: return launch_gs_mt<32>(st, pdl, g.grid, tm, g.p);
-    case 64: return launch_gs_mt<64>(st, pdl, g.grid, tm, g.p);
-    default: return launch_gs_mt<128>(st, pdl, g.grid, tm, g.p);
+    case 16: return deep ? launch_gs_mt<16, 1>(st, pdl, g.grid, tm, g.p) : launch_gs_mt<16, 0>(st, pdl, g.grid, tm, g.p);
+    case 32: return deep ? launch_gs_mt<32, 1>(st, pdl, g.grid, tm, g.p) : launch_gs_mt<32, 0>(st, pdl, g.grid, tm, g.p);
+    case 64: return deep ? launch_gs_mt<64, 1>(st, pdl, g.grid, tm, g.p) : launch_gs_mt<64, 0>(st, pdl, g.grid, tm, g.p);
+    default: return deep ? launch_gs_mt<128, 1>(st, pdl, g.grid, tm, g.p) : launch_gs_mt<128, 0>(st, pdl, g.grid, tm, g.p);
   }
 }
 
 PartView plan_view(const GemmPlan& g) {
   PartView v{};
-  v.part = g.p.part; v.slot_stride = g.p.slot_stride; v.ld = g.p.n_tiles * 128; v.seg = g.p.seg; v.MT = g.MT;
+  v.part = g.p.part; v.slot_stride = g.p.slot_stride; v.ld = g.p.n_tiles * 128; v.seg = g.p.seg;
+  v.mt_shift = g.MT == 16 ? 4 : (g.MT == 32 ? 5 : (g.MT == 64 ? 6 : 7));
   return v;
 }
 
@@ -175,7 +180,7 @@ struct spec_ctx {
   bool qkv_fused, keep_logits;
   bool pdl = true;                     // programmatic dependent launch between the kernels of a step
   int gemm_ctas = SM_SLOTS;            // persistent CTAs of the weight-streaming GEMM
-  int l2_prefetch = 8;                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
+  int l2_prefetch = 0;                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
   std::vector<int> h_parent, h_depth, h_rank;
   std::vector<int> n_hi;               // host upper bound of committed lengths
   std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, mw, mb;
@@ -195,6 +200,17 @@ struct spec_ctx {
   size_t part_floats;
   std::map<std::tuple<const void*, uint64_t, uint64_t, uint32_t>, CUtensorMap> tmaps;
   long long launches = 0;
+  // optional device timeline of the last step: four stamps per launch (see KTrace)
+  bool trace_on = false;
+  unsigned long long* d_trace = nullptr;
+  int trace_n = 0;
+  std::vector<std::string> trace_names;
+  std::vector<unsigned long long> trace_init;
+  unsigned long long* next_trace(const char* name) {
+    if (!trace_on || trace_n >= TRACE_CAP) return nullptr;
+    trace_names.push_back(name);
+    return d_trace + 4 * (size_t)(trace_n++);
+  }
   bool prefilled = false;
   // timing: phase boundaries of the last step; optional per-launch timing of one kernel kind
   cudaEvent_t phase_ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -277,6 +293,7 @@ size_t carve(spec_ctx* c, void* base) {
   size_t M = c->Mcap;
 
   c->d_status = b.take<int>(4);
+  c->d_trace = b.take<unsigned long long>((size_t)TRACE_CAP * 4);
   c->d_n = b.take<int>(B); c->d_cnt = b.take<int>(B); c->d_n_old = b.take<int>(B); c->d_root = b.take<int>(B);
   c->d_count = b.take<int>(B); c->d_path = b.take<int>((size_t)B * (K + 1)); c->d_out_tok = b.take<int>((size_t)B * (K + 1));
   c->d_gen_cnt = b.take<int>(B); c->d_gen_log = b.take<int>((size_t)B * c->gen_cap);
@@ -369,6 +386,16 @@ Rows make_rows(spec_ctx* c, int R, bool chain) {
   return r;
 }
 
+const char* gemm_kind_name(int kind) {
+  switch (kind) {
+    case SPEC_PROFILE_GATE_UP: return "gemm_gate_up";
+    case SPEC_PROFILE_QKV: return "gemm_qkv";
+    case SPEC_PROFILE_WO: return "gemm_wo";
+    case SPEC_PROFILE_DOWN: return "gemm_down";
+    default: return "gemm";
+  }
+}
+
 // ---- tensor-core linear (bf16): partial sums of x[M,K] * [mats]^T ----
 // kind: SPEC_PROFILE_* of the call site. On success *view describes the partial sums.
 int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* const* mats, const int* rows, int kind,
@@ -389,6 +416,7 @@ int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* c
   g.p.slot_stride = (size_t)M * g.p.n_tiles * 128;
   g.p.l2_prefetch = c->l2_prefetch;
   g.p.status = c->d_status;
+  g.p.trace = c->next_trace(gemm_kind_name(kind));
   {
     ProfScope ps(c, kind);
     cudaError_t e = launch_gs(c->stream, c->pdl, g, tm);
@@ -410,7 +438,7 @@ int linear_simple(spec_ctx* c, const T* x, int ldx, const T* W, float* y, int ld
 
 #define KLAUNCH(name, kernel, grid, block, smem, ...)                                            \
   do {                                                                                         \
-    cudaError_t e_ = launch_k(c->pdl, kernel, grid, block, smem, c->stream, __VA_ARGS__);      \
+    cudaError_t e_ = launch_k(c->pdl, kernel, grid, block, smem, c->stream, __VA_ARGS__, c->next_trace(name)); \
     c->launches++;                                                                             \
     if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string(name) + ": " + cudaGetErrorString(e_)); \
   } while (0)
@@ -457,52 +485,49 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain) {
   const int M = c->B * R, d = f.d_model, F = f.d_ffn, H = f.n_heads, D = f.head_dim, HD = H * D, KD = f.n_kv_heads * D;
   bf16* u = static_cast<bf16*>(c->d_u);
   bf16* act = static_cast<bf16*>(c->d_act);
-  const int tiles = 128;
-  const int kp0 = (HD + tiles - 1) / tiles * tiles, vp0 = kp0 + (KD + tiles - 1) / tiles * tiles;
-  const int up0 = (F + tiles - 1) / tiles * tiles;
+  const int kp0 = (HD + 127) / 128 * 128, vp0 = kp0 + (KD + 127) / 128 * 128;   // padded columns of k and v in the QKV partials
+  const int up0 = (F + 127) / 128 * 128;                                        // and of the up projection
+#define NORM_LAUNCH(pv, gain, uq, hid)                                                                   \
+  KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M), dim3(NORM_THREADS), 0, c->d_x, pv, gain, f.rms_eps, uq, hid, d)
   PartView pend{};              // partial sums of the previous down-projection still to be added to x
   for (int l = 0; l < f.n_layers; ++l) {
-    KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M), dim3(NORM_THREADS), 0, c->d_x, pend, c->an[l], f.rms_eps, u, (float*)nullptr, d);
+    NORM_LAUNCH(pend, c->an[l], u, (float*)nullptr);
+    int r;
     PartView vq{};
     {
       const void* mats[3] = {c->wq[l], c->wk[l], c->wv[l]};
       int rws[3] = {HD, KD, KD};
-      int r = run_gemm(c, u, M, d, 3, mats, rws, SPEC_PROFILE_QKV, &vq);
-      if (r) return r;
+      if ((r = run_gemm(c, u, M, d, 3, mats, rws, SPEC_PROFILE_QKV, &vq))) return r;
     }
-    KLAUNCH("rope_store_tc", rope_store_tc, dim3(M), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope, static_cast<bf16*>(c->d_q),
-            static_cast<bf16*>(c->d_pool), c->geom, c->d_page_table, l, H);
-    int r = launch_attention_tc(c, rows, R, l);
-    if (r) return r;
+    KLAUNCH("rope_store_tc", rope_store_tc, dim3(M, M <= 128 ? 4 : 1), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope,
+            static_cast<bf16*>(c->d_q), static_cast<bf16*>(c->d_pool), c->geom, c->d_page_table, l, H);
+    if ((r = launch_attention_tc(c, rows, R, l))) return r;
     PartView vo{};
     {
       const void* mats[1] = {c->wo[l]};
       int rws[1] = {d};
-      r = run_gemm(c, c->d_attn, M, HD, 1, mats, rws, SPEC_PROFILE_WO, &vo);
-      if (r) return r;
+      if ((r = run_gemm(c, c->d_attn, M, HD, 1, mats, rws, SPEC_PROFILE_WO, &vo))) return r;
     }
-    KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M), dim3(NORM_THREADS), 0, c->d_x, vo, c->fn[l], f.rms_eps, u, (float*)nullptr, d);
+    NORM_LAUNCH(vo, c->fn[l], u, (float*)nullptr);
     PartView vg{};
     {
       const void* mats[2] = {c->wg[l], c->wu[l]};
       int rws[2] = {F, F};
-      r = run_gemm(c, u, M, d, 2, mats, rws, SPEC_PROFILE_GATE_UP, &vg);
-      if (r) return r;
+      if ((r = run_gemm(c, u, M, d, 2, mats, rws, SPEC_PROFILE_GATE_UP, &vg))) return r;
     }
     {
       size_t total = (size_t)M * (F / 4);
-      unsigned blocks = (unsigned)std::min<size_t>((total + 255) / 256, 2048);
+      unsigned blocks = (unsigned)std::min<size_t>((total + 255) / 256, 2 * SM_SLOTS);
       KLAUNCH("swiglu_reduce_tc", swiglu_reduce_tc, dim3(blocks), dim3(256), 0, vg, 0, up0, act, M, F);
     }
     {
       const void* mats[1] = {c->wd[l]};
       int rws[1] = {d};
-      r = run_gemm(c, act, M, F, 1, mats, rws, SPEC_PROFILE_DOWN, &pend);
-      if (r) return r;
+      if ((r = run_gemm(c, act, M, F, 1, mats, rws, SPEC_PROFILE_DOWN, &pend))) return r;
     }
   }
-  KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M), dim3(NORM_THREADS), 0, c->d_x, pend, c->final_norm, f.rms_eps,
-          static_cast<bf16*>(c->d_hq), c->d_hid, d);
+  NORM_LAUNCH(pend, c->final_norm, static_cast<bf16*>(c->d_hq), c->d_hid);
+#undef NORM_LAUNCH
   return SPEC_OK;
 }
 
@@ -572,6 +597,7 @@ int lm_head_argmax(spec_ctx* c, const T* src, int M) {
     g.p.pval = c->d_pval; g.p.pidx = c->d_pidx;
     g.p.l2_prefetch = c->l2_prefetch;
     g.p.status = c->d_status;
+    g.p.trace = c->next_trace("gemm_lm_head");
     cudaError_t e = launch_gs(c->stream, c->pdl, g, tm);
     c->launches++;
     if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_stream lm_head launch: ") + cudaGetErrorString(e));
@@ -661,6 +687,11 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   for (int i = 0; i < 6; ++i)
     if (!c->phase_ev[i]) CUDA_OK(cudaEventCreate(&c->phase_ev[i]));
   c->prof_used = 0;
+  if (c->trace_on) {
+    c->trace_n = 0;
+    c->trace_names.clear();
+    CUDA_OK(cudaMemcpyAsync(c->d_trace, c->trace_init.data(), c->trace_init.size() * 8, cudaMemcpyHostToDevice, c->stream));
+  }
   cudaEventRecord(c->phase_ev[0], c->stream);
   const int* ov = nullptr;
   if (cand_override && K > 0) {
@@ -671,19 +702,17 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   if (K > 0) {
     constexpr int MC = 4;
     dim3 g1((K * d + 7) / 8, (B + MC - 1) / MC);
-    medusa_resblock<T, MC><<<g1, 256, 0, c->stream>>>(c->d_h_last, reinterpret_cast<const T* const*>(c->d_mw),
-                                                    reinterpret_cast<const T* const*>(c->d_mb), static_cast<T*>(c->d_r), B, K, d);
-    LAUNCH_CHECK("medusa_resblock");
+    KLAUNCH("medusa_resblock", (medusa_resblock<T, MC>), g1, dim3(256), 0, (const float*)c->d_h_last,
+            reinterpret_cast<const T* const*>(c->d_mw), reinterpret_cast<const T* const*>(c->d_mb), static_cast<T*>(c->d_r), B, K, d);
     int rows_total = B * K;
     dim3 g2(c->topk_blocks, (rows_total + MC - 1) / MC);
     size_t sm = (size_t)MC * c->topk_slice * sizeof(float);
-    medusa_lmhead_topk<T, MC><<<g2, 256, sm, c->stream>>>(static_cast<const T*>(c->d_r), static_cast<const T*>(c->lm_head), rows_total,
-                                                        f.vocab, d, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
-    LAUNCH_CHECK("medusa_lmhead_topk");
+    KLAUNCH("medusa_lmhead_topk", (medusa_lmhead_topk<T, MC>), g2, dim3(256), sm, static_cast<const T*>(c->d_r),
+            static_cast<const T*>(c->lm_head), rows_total, f.vocab, d, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
     // partial lists of the row chunks are laid out per block over all rows
     size_t sm2 = (size_t)c->topk_blocks * kmax * 8;
-    topk_merge<<<rows_total, 256, sm2, c->stream>>>(c->d_pk_val, c->d_pk_idx, c->topk_blocks, rows_total, K, kmax, c->d_root, ov, c->d_cand);
-    LAUNCH_CHECK("topk_merge");
+    KLAUNCH("topk_merge", topk_merge, dim3(rows_total), dim3(256), sm2, (const float*)c->d_pk_val, (const int*)c->d_pk_idx,
+            c->topk_blocks, rows_total, K, kmax, (const int*)c->d_root, ov, c->d_cand);
   } else {
     CUDA_OK(cudaMemcpyAsync(c->d_cand, c->d_root, B * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
   }
@@ -691,9 +720,8 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   // (2) candidate tree -> rows
   int M = B * T_;
   Rows rows = make_rows(c, T_, false);
-  prepare_verify_rows<T><<<M, 128, 0, c->stream>>>(rows, c->d_cand, (K + 1) * kmax, kmax, c->d_depth, c->d_rank, c->cap,
-                                                 static_cast<const T*>(c->embed), c->d_x, d, f.vocab, c->d_status);
-  LAUNCH_CHECK("prepare_verify_rows");
+  KLAUNCH("prepare_verify_rows", prepare_verify_rows<T>, dim3(M), dim3(128), 0, rows, (const int*)c->d_cand, (K + 1) * kmax, kmax,
+          (const int*)c->d_depth, (const int*)c->d_rank, c->cap, static_cast<const T*>(c->embed), c->d_x, d, f.vocab, c->d_status);
   cudaEventRecord(c->phase_ev[2], c->stream);
   // (3) verification forward
   int r = forward_layers<T>(c, T_, false);
@@ -713,8 +741,8 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   cudaEventRecord(c->phase_ev[4], c->stream);
   // (5) KV compaction
   dim3 gc(f.n_layers * 2 * f.n_kv_heads, B);
-  compact_kv<T><<<gc, 64, 0, c->stream>>>(static_cast<T*>(c->d_pool), c->geom, c->d_page_table, c->d_path, c->d_count, c->d_n_old, K);
-  LAUNCH_CHECK("compact_kv");
+  KLAUNCH("compact_kv", compact_kv<T>, gc, dim3(64), 0, static_cast<T*>(c->d_pool), c->geom, (const int*)c->d_page_table,
+          (const int*)c->d_path, (const int*)c->d_count, (const int*)c->d_n_old, K);
   cudaEventRecord(c->phase_ev[5], c->stream);
   c->phase_valid = true;
   if (c->profile_kind) {
@@ -911,8 +939,31 @@ int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
     case SPEC_OPT_L2_PREFETCH:
       if (value < 0 || value > 64) return c->fail(SPEC_E_BADARG, "L2 prefetch depth out of range");
       c->l2_prefetch = value; return SPEC_OK;
+    case SPEC_OPT_TRACE:
+      c->trace_on = value != 0;
+      if (c->trace_on && c->trace_init.empty()) {
+        c->trace_init.resize((size_t)TRACE_CAP * 4);
+        for (int i = 0; i < TRACE_CAP; ++i) { c->trace_init[4 * i] = ~0ull; c->trace_init[4 * i + 1] = 0; c->trace_init[4 * i + 2] = ~0ull; c->trace_init[4 * i + 3] = 0; }
+      }
+      return SPEC_OK;
     default: return c->fail(SPEC_E_BADARG, "unknown option");
   }
+}
+
+int spec_trace_read(spec_ctx* c, int32_t max_records, char* names, uint64_t* stamps, int32_t* n_records) {
+  if (!c || !n_records || max_records < 0 || (max_records > 0 && (!names || !stamps))) return SPEC_E_BADARG;
+  if (!c->trace_on) return c->fail(SPEC_E_STATE, "tracing is off (SPEC_OPT_TRACE)");
+  int n = c->trace_n < max_records ? c->trace_n : max_records;
+  if (n > 0) {
+    CUDA_OK(cudaMemcpyAsync(stamps, c->d_trace, (size_t)n * 32, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_OK(cudaStreamSynchronize(c->stream));
+    for (int i = 0; i < n; ++i) {
+      strncpy(names + (size_t)i * SPEC_TRACE_NAME_LEN, c->trace_names[i].c_str(), SPEC_TRACE_NAME_LEN - 1);
+      names[(size_t)i * SPEC_TRACE_NAME_LEN + SPEC_TRACE_NAME_LEN - 1] = 0;
+    }
+  }
+  *n_records = c->trace_n;
+  return SPEC_OK;
 }
 
 int spec_last_step_phase_ms(spec_ctx* c, float* ms) {
