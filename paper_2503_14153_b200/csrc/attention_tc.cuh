@@ -1,12 +1,17 @@
 // Tree-masked decode attention over the paged bf16 KV cache (verification forward of
 // Sec. III-B: every tree node attends to all committed positions and to its own ancestors
-// in the tree). One CTA per (query head, KV split, sequence); warp w owns query rows
-// [16w, 16w+16). KV tiles of 64 keys are brought in page by page with bulk asynchronous
+// in the tree). One CTA per (query head, KV split, sequence) with NW x KG warps: warp
+// (rg, kg) owns query rows [16 rg, 16 rg + 16) and every KG-th tile of the split, so two
+// tiles are worked on at a time; the key groups' softmax states are merged through shared
+// memory at the end. KV tiles of 64 keys are brought in page by page with bulk asynchronous
 // copies that complete on an mbarrier (the cache's in-page chunk swizzle makes the landed
 // tile conflict-free for ldmatrix); QK^T and PV run on mma.sync m16n8k16 with a warp-level
 // online softmax; the tree mask is a 128-bit ancestor set per row applied only to keys at or
-// beyond the committed length. Each split leaves (max, sum, unnormalised output) and a
-// small combine kernel merges the splits.
+// beyond the committed length. The host picks the number of KV splits from its bound on the
+// context length; tiles that hold only rows of earlier steps are fetched before the wait on
+// the previous kernel. With one split the CTA writes the normalised bf16 output
+// itself, otherwise each split leaves (max, sum, unnormalised output) and the CTA of a
+// (sequence, head) that finishes last (arrival counter, no waiting) merges them.
 #pragma once
 #include "common.cuh"
 #include "kernels_simple.cuh"
@@ -14,15 +19,15 @@
 namespace spec {
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+  asm("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+  asm("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -32,6 +37,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+constexpr int ATTN_MAX_STAGES = 4;
+constexpr int ATTN_PT_CACHE = 256;
+constexpr int ATTN_MAX_SEQS = 16;
+
 struct AttnTcArgs {
   const bf16* q;        // [M][H*HD]
   float* part_o;        // [nsplit][M][H*HD] unnormalised
@@ -40,84 +49,142 @@ struct AttnTcArgs {
   KVGeom g;
   const int* page_table;
   Rows rows;
-  int layer, H, nsplit;
+  int layer, H;
+  int nsplit;           // KV splits (= gridDim.y), chosen by the host from its bound on the context length
+  int tps;              // KV tiles per split
+  int stages;           // KV tiles in flight per CTA (2..ATTN_MAX_STAGES, a multiple of KG); sizes the shared memory
+  int n_lo[ATTN_MAX_SEQS];   // host's lower bound of each sequence's committed length: keys below it
+                             // were written by earlier steps and may be fetched before the dependency wait
   float scale_log2;     // log2(e) / sqrt(head_dim)
+  bf16* out;            // [M][H*HD]
+  unsigned int* arrive; // [B][H] arrival counters, zero between launches
   int* status;
 };
 
-template <int HD, int NW>
-__global__ void __launch_bounds__(NW * 32)
+__host__ __device__ inline size_t attention_tc_smem(int head_dim, int nw, int stages) {
+  const size_t rowb = (size_t)head_dim * 2;
+  return (size_t)nw * 16 * rowb + 2 * (size_t)stages * 64 * rowb + 8 * ATTN_MAX_STAGES + 4 * ATTN_PT_CACHE;
+}
+
+// 64 visibility bits of one query row for keys k0 .. k0+63: keys below the committed length n
+// are visible, key n + u is visible iff bit u of the row's 128-bit ancestor set is set.
+__device__ __forceinline__ unsigned long long attn_vis64(const uint32_t (&an)[4], int k0, int n) {
+  const int u0 = k0 - n;
+  const unsigned long long A0 = an[0] | ((unsigned long long)an[1] << 32), A1 = an[2] | ((unsigned long long)an[3] << 32);
+  if (u0 <= -64) return ~0ull;
+  if (u0 < 0) return ((1ull << (-u0)) - 1ull) | (A0 << (-u0));
+  if (u0 == 0) return A0;
+  if (u0 < 64) return (A0 >> u0) | (A1 << (64 - u0));
+  if (u0 == 64) return A1;
+  if (u0 < 128) return A1 >> (u0 - 64);
+  return 0ull;
+}
+
+template <int HD, int NW, int KG>
+__global__ void __launch_bounds__(NW * KG * 32)
 attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   KTrace kt(tr);
   constexpr int KT = 64;                      // keys per tile
   constexpr int ROWB = HD * 2;                // bytes per row
   constexpr int TILE_BYTES = KT * ROWB;
   constexpr int PAGE_BYTES = 16 * ROWB;
+  constexpr int NTHR = NW * KG * 32;
+  const int ST = a.stages;
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* qs = smem;                                       // [NW*16][HD]
-  uint8_t* ks = qs + NW * 16 * ROWB;                        // [2][KT][HD]
-  uint8_t* vs = ks + 2 * TILE_BYTES;                        // [2][KT][HD]
-  uint64_t* full = reinterpret_cast<uint64_t*>(vs + 2 * TILE_BYTES);   // [2]
+  uint8_t* ks = qs + NW * 16 * ROWB;                        // [ST][KT][HD]
+  uint8_t* vs = ks + ST * TILE_BYTES;                       // [ST][KT][HD]
+  uint64_t* full = reinterpret_cast<uint64_t*>(vs + ST * TILE_BYTES);   // [ATTN_MAX_STAGES]
+  int* pt_s = reinterpret_cast<int*>(full + ATTN_MAX_STAGES);           // [ATTN_PT_CACHE] page-table entries of this split
 
   pdl_launch_dependents();
-  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rg = warp % NW, kg = warp / NW;
   const int h = blockIdx.x, sp = blockIdx.y, b = blockIdx.z;
-  const int R = a.rows.R, cnt = a.rows.cnt[b], n = a.rows.n[b];
-  const int S = n + cnt;
   const int H = a.H, kvh = h / (H / a.g.n_kv_heads);
-  const int M = a.rows.B * R;
-  if (cnt == 0) return;
-  const int total_tiles = (S + KT - 1) / KT;
-  const int tps = (total_tiles + a.nsplit - 1) / a.nsplit;
-  const int t0 = sp * tps, t1 = min(total_tiles, t0 + tps);
+  const int nsplit = a.nsplit, tps = a.tps;
+  const int t0 = sp * tps;
   const int* pt = a.page_table + b * a.g.pages_per_seq;
-
-  const int i0 = warp * 16 + (lane >> 2), i1 = i0 + 8;      // this thread's two query rows
-  if (t0 >= t1) {
-    // empty split: publish a neutral partial for the valid rows
-    if ((lane & 3) == 0) {
-      if (i0 < cnt) { float* ml = a.part_ml + (((size_t)sp * M + b * R + i0) * H + h) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
-      if (i1 < cnt) { float* ml = a.part_ml + (((size_t)sp * M + b * R + i1) * H + h) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
-    }
-    return;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < ST; ++i) mbar_init(&full[i], 1);
+    mbar_fence_init();
   }
-
-  if (threadIdx.x == 0) { mbar_init(&full[0], 1); mbar_init(&full[1], 1); mbar_fence_init(); }
-  // stage Q (rows beyond cnt are zero) with the same chunk swizzle as the cache
-  for (int c = threadIdx.x; c < NW * 16 * (HD / 8); c += NW * 32) {
-    int r = c / (HD / 8), ch = c % (HD / 8);
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (r < cnt) v = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + r) * H * HD + h * HD + ch * 8);
-    *reinterpret_cast<uint4*>(qs + r * ROWB + ((ch ^ (r & 7)) << 4)) = v;
+  // the page table is fixed at set-up: stage this split's entries before the dependency wait
+  for (int e = threadIdx.x; e < tps * (KT / 16) && e < ATTN_PT_CACHE; e += NTHR) {
+    const int idx = t0 * (KT / 16) + e;
+    pt_s[e] = idx < a.g.pages_per_seq ? pt[idx] : 0;
   }
-  __syncthreads();
-
+  __syncthreads();   // barriers initialised, page entries staged
   auto issue = [&](int tile, int buf) {
     mbar_expect_tx(&full[buf], 2 * TILE_BYTES);
     for (int pg = 0; pg < KT / 16; ++pg) {
-      int page = pt[tile * (KT / 16) + pg];
+      const int e = (tile - t0) * (KT / 16) + pg;
+      const int page = e < ATTN_PT_CACHE ? pt_s[e] : pt[tile * (KT / 16) + pg];
       bulk_load_1d(ks + buf * TILE_BYTES + pg * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 0, kvh),
                    PAGE_BYTES, &full[buf]);
       bulk_load_1d(vs + buf * TILE_BYTES + pg * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 1, kvh),
                    PAGE_BYTES, &full[buf]);
     }
   };
-  if (threadIdx.x == 0) issue(t0, 0);
+  // tiles that lie wholly below the host's lower bound of the committed length hold rows of
+  // earlier steps: start fetching them now (thread 0 keeps the count)
+  int pre = 0;
+  if (threadIdx.x == 0) {
+    const int safe = (b < ATTN_MAX_SEQS ? a.n_lo[b] : 0) / KT;      // tiles [0, safe) are committed
+    const int lim = min(t0 + tps, safe);
+    for (; pre < ST && t0 + pre < lim; ++pre) issue(t0 + pre, pre);
+  }
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  const int R = a.rows.R, cnt = a.rows.cnt[b], n = a.rows.n[b];
+  const int S = n + cnt;
+  const int M = a.rows.B * R;
+  const int total_tiles = (S + KT - 1) / KT;
+  const int t1 = min(total_tiles, t0 + tps);
+  const int i0 = rg * 16 + (lane >> 2), i1 = i0 + 8;        // this thread's two query rows
+  if (cnt == 0) {
+    // inactive sequence: let the copies already in flight land before the CTA goes away
+    if (threadIdx.x == 0)
+      for (int i = 0; i < pre; ++i) mbar_wait(&full[i], 0, a.status, 21);
+    return;
+  }
+  // the rest of the first tiles
+  if (threadIdx.x == 0)
+    for (int i = pre; i < ST && t0 + i < t1; ++i) issue(t0 + i, i);
+  // ancestor sets and Q (rows beyond cnt are zero): all loads first, then the swizzled stores
+  uint32_t anc0[4] = {0, 0, 0, 0}, anc1[4] = {0, 0, 0, 0};
+  if (i0 < cnt) for (int w = 0; w < 4; ++w) anc0[w] = a.rows.anc[i0 * 4 + w];
+  if (i1 < cnt) for (int w = 0; w < 4; ++w) anc1[w] = a.rows.anc[i1 * 4 + w];
+  {
+    constexpr int QC = NW * 16 * (HD / 8);                    // 16-byte chunks of the Q tile
+    constexpr int PER = (QC + NTHR - 1) / NTHR;
+    uint4 qv[PER];
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      const int c = threadIdx.x + k * NTHR;
+      const int r = c / (HD / 8), ch = c % (HD / 8);
+      qv[k] = make_uint4(0, 0, 0, 0);
+      if (c < QC && r < cnt) qv[k] = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + r) * H * HD + h * HD + ch * 8);
+    }
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      const int c = threadIdx.x + k * NTHR;
+      const int r = c / (HD / 8), ch = c % (HD / 8);
+      if (c < QC) *reinterpret_cast<uint4*>(qs + r * ROWB + ((ch ^ (r & 7)) << 4)) = qv[k];
+    }
+  }
+  __syncthreads();
 
   // Q fragments stay in registers
   uint32_t qf[HD / 16][4];
   {
-    int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    int row = rg * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
     for (int kk = 0; kk < HD / 16; ++kk) {
       int ch = kk * 2 + (lane >> 4);
       ldmatrix_x4(smem_u32(qs + row * ROWB + ((ch ^ (row & 7)) << 4)), qf[kk]);
     }
   }
-  uint32_t anc0[4] = {0, 0, 0, 0}, anc1[4] = {0, 0, 0, 0};
-  if (i0 < cnt) for (int w = 0; w < 4; ++w) anc0[w] = a.rows.anc[i0 * 4 + w];
-  if (i1 < cnt) for (int w = 0; w < 4; ++w) anc1[w] = a.rows.anc[i1 * 4 + w];
 
   float o[HD / 8][4];
 #pragma unroll
@@ -125,97 +192,172 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
 
   bool ok = true;
-  for (int t = t0; t < t1; ++t) {
-    const int buf = (t - t0) & 1;
-    if (threadIdx.x == 0 && t + 1 < t1) issue(t + 1, buf ^ 1);
-    if (!mbar_wait(&full[buf], ((t - t0) >> 1) & 1, a.status, 20)) { ok = false; }
+  const int ntile = t1 - t0;
+  for (int it = 0; it < ntile; it += KG) {
+    const int my = it + kg;                 // this warp's tile of the round, relative to t0
+    const bool have = my < ntile;
+    if (have && !mbar_wait(&full[my % ST], (my / ST) & 1, a.status, 20)) ok = false;
     ok = __syncthreads_and(ok);
     if (!ok) break;
-    const uint8_t* kt = ks + buf * TILE_BYTES;
-    const uint8_t* vt = vs + buf * TILE_BYTES;
-    float s[KT / 8][4];
+    if (it == 0 && threadIdx.x == 0) trace_mark_max(tr, 3);
+    if (have) {
+      const int t = t0 + my;
+      const uint8_t* kt = ks + (my % ST) * TILE_BYTES;
+      const uint8_t* vt = vs + (my % ST) * TILE_BYTES;
+      float s[KT / 8][4];
 #pragma unroll
-    for (int j = 0; j < KT / 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+      for (int j = 0; j < KT / 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+      // K fragments of a 16-wide slice of the head dimension are fetched together, one slice
+      // ahead of the MMAs that use them
+      {
+        uint32_t kf[2][KT / 16][4];
+        auto load_k = [&](int kk, uint32_t (&dst)[KT / 16][4]) {
 #pragma unroll
-    for (int kk = 0; kk < HD / 16; ++kk) {
-#pragma unroll
-      for (int j2 = 0; j2 < KT / 16; ++j2) {
-        int key = j2 * 16 + (lane & 7) + (lane >> 4) * 8;
-        int ch = kk * 2 + ((lane >> 3) & 1);
-        uint32_t bfr[4];
-        ldmatrix_x4(smem_u32(kt + key * ROWB + ((ch ^ (key & 7)) << 4)), bfr);
-        mma_bf16_16816(s[2 * j2], qf[kk], bfr[0], bfr[1]);
-        mma_bf16_16816(s[2 * j2 + 1], qf[kk], bfr[2], bfr[3]);
-      }
-    }
-    // mask + online softmax (log2 domain)
-    const int k0 = t * KT;
-    const bool need_mask = (k0 + KT > n);
-    float tmax[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-    for (int j = 0; j < KT / 8; ++j) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float v = s[j][e] * a.scale_log2;
-        if (need_mask) {
-          int key = k0 + j * 8 + (lane & 3) * 2 + (e & 1);
-          bool vis = key < n;
-          if (!vis && key < S) {
-            int u = key - n;
-            uint32_t w = (e < 2) ? anc0[u >> 5] : anc1[u >> 5];
-            vis = (w >> (u & 31)) & 1u;
+          for (int j2 = 0; j2 < KT / 16; ++j2) {
+            int key = j2 * 16 + (lane & 7) + (lane >> 4) * 8;
+            int ch = kk * 2 + ((lane >> 3) & 1);
+            ldmatrix_x4(smem_u32(kt + key * ROWB + ((ch ^ (key & 7)) << 4)), dst[j2]);
           }
-          if (!vis) v = -INFINITY;
+        };
+        load_k(0, kf[0]);
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          if (kk + 1 < HD / 16) load_k(kk + 1, kf[(kk + 1) & 1]);
+#pragma unroll
+          for (int j2 = 0; j2 < KT / 16; ++j2) {
+            mma_bf16_16816(s[2 * j2], qf[kk], kf[kk & 1][j2][0], kf[kk & 1][j2][1]);
+            mma_bf16_16816(s[2 * j2 + 1], qf[kk], kf[kk & 1][j2][2], kf[kk & 1][j2][3]);
+          }
         }
-        s[j][e] = v;
-        tmax[e >> 1] = fmaxf(tmax[e >> 1], v);
+      }
+      // mask + online softmax (log2 domain)
+      const int k0 = t * KT;
+      const bool need_mask = (k0 + KT > n);
+      unsigned long long vis0 = ~0ull, vis1 = ~0ull;
+      if (need_mask) { vis0 = attn_vis64(anc0, k0, n); vis1 = attn_vis64(anc1, k0, n); }
+      float tmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+      for (int j = 0; j < KT / 8; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float v = s[j][e] * a.scale_log2;
+          const int bi = j * 8 + (lane & 3) * 2 + (e & 1);
+          if (!(((e < 2 ? vis0 : vis1) >> bi) & 1ull)) v = -INFINITY;
+          s[j][e] = v;
+          tmax[e >> 1] = fmaxf(tmax[e >> 1], v);
+        }
+      }
+      float alpha[2], mnew[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 1));
+        tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 2));
+        mnew[r] = fmaxf(mrow[r], tmax[r]);
+        float base = (mnew[r] == -INFINITY) ? 0.f : mnew[r];
+        alpha[r] = exp2f(mrow[r] - base);
+        mrow[r] = mnew[r];
+        mnew[r] = base;
+        lrow[r] *= alpha[r];
+      }
+#pragma unroll
+      for (int d = 0; d < HD / 8; ++d) { o[d][0] *= alpha[0]; o[d][1] *= alpha[0]; o[d][2] *= alpha[1]; o[d][3] *= alpha[1]; }
+      uint32_t pf[KT / 16][4];
+#pragma unroll
+      for (int j = 0; j < KT / 8; ++j) {
+        float p0 = exp2f(s[j][0] - mnew[0]), p1 = exp2f(s[j][1] - mnew[0]);
+        float p2 = exp2f(s[j][2] - mnew[1]), p3 = exp2f(s[j][3] - mnew[1]);
+        lrow[0] += p0 + p1;
+        lrow[1] += p2 + p3;
+        pf[j >> 1][(j & 1) * 2 + 0] = pack_bf16(p0, p1);
+        pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
+      }
+      // V fragments: four 16-wide slices of the head dimension at a time, one group ahead
+      {
+        constexpr int DG = 4, NG = (KT / 16) * (HD / 16) / DG;
+        uint32_t vf[2][DG][4];
+        auto load_v = [&](int g, uint32_t (&dst)[DG][4]) {
+          const int j = g / (HD / 16 / DG), d0 = (g % (HD / 16 / DG)) * DG;
+#pragma unroll
+          for (int dd = 0; dd < DG; ++dd) {
+            int key = j * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            int ch = (d0 + dd) * 2 + (lane >> 4);
+            ldmatrix_x4_trans(smem_u32(vt + key * ROWB + ((ch ^ (key & 7)) << 4)), dst[dd]);
+          }
+        };
+        load_v(0, vf[0]);
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          if (g + 1 < NG) load_v(g + 1, vf[(g + 1) & 1]);
+          const int j = g / (HD / 16 / DG), d0 = (g % (HD / 16 / DG)) * DG;
+#pragma unroll
+          for (int dd = 0; dd < DG; ++dd) {
+            mma_bf16_16816(o[2 * (d0 + dd)], pf[j], vf[g & 1][dd][0], vf[g & 1][dd][1]);
+            mma_bf16_16816(o[2 * (d0 + dd) + 1], pf[j], vf[g & 1][dd][2], vf[g & 1][dd][3]);
+          }
+        }
       }
     }
-    float alpha[2], mnew[2];
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 1));
-      tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 2));
-      mnew[r] = fmaxf(mrow[r], tmax[r]);
-      float base = (mnew[r] == -INFINITY) ? 0.f : mnew[r];
-      alpha[r] = exp2f(mrow[r] - base);
-      mrow[r] = mnew[r];
-      mnew[r] = base;
-      lrow[r] *= alpha[r];
-    }
-#pragma unroll
-    for (int d = 0; d < HD / 8; ++d) { o[d][0] *= alpha[0]; o[d][1] *= alpha[0]; o[d][2] *= alpha[1]; o[d][3] *= alpha[1]; }
-    uint32_t pf[KT / 16][4];
-#pragma unroll
-    for (int j = 0; j < KT / 8; ++j) {
-      float p0 = exp2f(s[j][0] - mnew[0]), p1 = exp2f(s[j][1] - mnew[0]);
-      float p2 = exp2f(s[j][2] - mnew[1]), p3 = exp2f(s[j][3] - mnew[1]);
-      lrow[0] += p0 + p1;
-      lrow[1] += p2 + p3;
-      pf[j >> 1][(j & 1) * 2 + 0] = pack_bf16(p0, p1);
-      pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
-    }
-#pragma unroll
-    for (int j = 0; j < KT / 16; ++j) {
-#pragma unroll
-      for (int d2 = 0; d2 < HD / 16; ++d2) {
-        int key = j * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        int ch = d2 * 2 + (lane >> 4);
-        uint32_t bfr[4];
-        ldmatrix_x4_trans(smem_u32(vt + key * ROWB + ((ch ^ (key & 7)) << 4)), bfr);
-        mma_bf16_16816(o[2 * d2], pf[j], bfr[0], bfr[1]);
-        mma_bf16_16816(o[2 * d2 + 1], pf[j], bfr[2], bfr[3]);
-      }
-    }
-    __syncthreads();   // tile consumed: its buffer may be refilled
+    __syncthreads();   // the round's tiles are consumed: their buffers may be refilled
+    if (threadIdx.x == 0)
+      for (int g = 0; g < KG; ++g)
+        if (it + g + ST < ntile) issue(t0 + it + g + ST, (it + g) % ST);
   }
+  if (!ok) return;
 
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
     lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
     lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
   }
-  if (ok) {
+  if (KG == 2) {
+    // merge the two key groups' states through the (now idle) KV buffers
+    float* ex = reinterpret_cast<float*>(ks);
+    constexpr int GT = NW * 32;                                // threads per key group
+    const int gt = rg * 32 + lane;
+    if (kg == 1) {
+#pragma unroll
+      for (int d = 0; d < HD / 8; ++d)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) ex[(d * 4 + e) * GT + gt] = o[d][e];
+      ex[(HD / 2 + 0) * GT + gt] = mrow[0]; ex[(HD / 2 + 1) * GT + gt] = mrow[1];
+      ex[(HD / 2 + 2) * GT + gt] = lrow[0]; ex[(HD / 2 + 3) * GT + gt] = lrow[1];
+    }
+    __syncthreads();
+    if (kg == 0) {
+      float w0[2], w1[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const float m1 = ex[(HD / 2 + r) * GT + gt], l1 = ex[(HD / 2 + 2 + r) * GT + gt];
+        const float mm = fmaxf(mrow[r], m1);
+        const float base = (mm == -INFINITY) ? 0.f : mm;
+        w0[r] = exp2f(mrow[r] - base);
+        w1[r] = exp2f(m1 - base);
+        mrow[r] = mm;
+        lrow[r] = lrow[r] * w0[r] + l1 * w1[r];
+      }
+#pragma unroll
+      for (int d = 0; d < HD / 8; ++d)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[d][e] = o[d][e] * w0[e >> 1] + ex[(d * 4 + e) * GT + gt] * w1[e >> 1];
+    }
+  }
+  if (nsplit == 1) {
+    // the only split: normalise and store the bf16 output
+    if (kg == 0) {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        int i = r ? i1 : i0;
+        if (i >= cnt) continue;
+        const float inv = 1.f / lrow[r];
+        bf16* po = a.out + ((size_t)b * R + i) * H * HD + h * HD;
+#pragma unroll
+        for (int d = 0; d < HD / 8; ++d)
+          *reinterpret_cast<uint32_t*>(po + d * 8 + (lane & 3) * 2) = pack_bf16(o[d][2 * r] * inv, o[d][2 * r + 1] * inv);
+      }
+    }
+    return;
+  }
+  if (kg == 0) {
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
       int i = r ? i1 : i0;
@@ -232,41 +374,66 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
       }
     }
   }
-}
-
-// Merges the KV splits: out[m][h*HD + d] = bf16( sum_s w_s O_s / sum_s w_s l_s ),
-// w_s = 2^(m_s - max_s m_s). One thread per (row, head, 4 dims).
-__global__ void attention_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml, int nsplit,
-                                  Rows rows, int H, int HD, bf16* __restrict__ out, unsigned long long* tr) {
-  KTrace kt(tr);
-  pdl_launch_dependents();
-  pdl_wait();
-  if (threadIdx.x == 0) trace_mark_min(tr, 2);
-  int M = rows.B * rows.R;
-  size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  size_t per_row = (size_t)H * HD / 4;
-  if (idx >= (size_t)M * per_row) return;
-  int m = (int)(idx / per_row);
-  int rem = (int)(idx % per_row);
-  int h = rem / (HD / 4), d = (rem % (HD / 4)) * 4;
-  if (m % rows.R >= rows.cnt[m / rows.R]) return;
-  float mx = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) mx = fmaxf(mx, part_ml[(((size_t)s * M + m) * H + h) * 2]);
-  float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int s = 0; s < nsplit; ++s) {
-    const float* ml = part_ml + (((size_t)s * M + m) * H + h) * 2;
-    if (ml[0] == -INFINITY) continue;
-    float w = exp2f(ml[0] - mx);
-    L += w * ml[1];
-    float4 v = *reinterpret_cast<const float4*>(part_o + ((size_t)s * M + m) * H * HD + h * HD + d);
-    acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
+  // the CTA of this (sequence, head) that arrives last merges the splits
+  __shared__ int last_s;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int old = atomicAdd(a.arrive + b * H + h, 1u);
+    const int last = (old == (unsigned int)(nsplit - 1)) ? 1 : 0;
+    if (last) a.arrive[b * H + h] = 0u;
+    last_s = last;
   }
-  float inv = 1.f / L;
-  bf16* o = out + (size_t)m * H * HD + h * HD + d;
-  o[0] = __float2bfloat16_rn(acc[0] * inv);
-  o[1] = __float2bfloat16_rn(acc[1] * inv);
-  o[2] = __float2bfloat16_rn(acc[2] * inv);
-  o[3] = __float2bfloat16_rn(acc[3] * inv);
+  __syncthreads();
+  if (!last_s) return;
+  __threadfence();
+  // two threads per query row, each merging half of the head dimension
+  {
+    const int i = threadIdx.x >> 1, d0 = (threadIdx.x & 1) * (HD / 2);
+    if (i < cnt && i < NW * 16) {
+      const size_t m = (size_t)b * R + i;
+      float wgt[16];
+      float mx = -INFINITY, L = 0.f;
+#pragma unroll
+      for (int s2 = 0; s2 < 16; ++s2) {
+        wgt[s2] = -INFINITY;
+        if (s2 < nsplit) wgt[s2] = __ldcg(a.part_ml + (((size_t)s2 * M + m) * H + h) * 2);
+        mx = fmaxf(mx, wgt[s2]);
+      }
+#pragma unroll
+      for (int s2 = 0; s2 < 16; ++s2)
+        if (s2 < nsplit) {
+          const float l2 = __ldcg(a.part_ml + (((size_t)s2 * M + m) * H + h) * 2 + 1);
+          wgt[s2] = exp2f(wgt[s2] - mx);
+          L += wgt[s2] * l2;
+        }
+      float acc[HD / 2];
+#pragma unroll
+      for (int e = 0; e < HD / 2; ++e) acc[e] = 0.f;
+#pragma unroll
+      for (int s2 = 0; s2 < 16; ++s2) {
+        if (s2 >= nsplit) break;
+        const float w = wgt[s2];
+        const float* src = a.part_o + ((size_t)s2 * M + m) * H * HD + h * HD + d0;
+        float4 v[HD / 8];
+#pragma unroll
+        for (int e = 0; e < HD / 8; ++e) v[e] = __ldcg(reinterpret_cast<const float4*>(src + e * 4));
+#pragma unroll
+        for (int e = 0; e < HD / 8; ++e) {
+          acc[4 * e] += w * v[e].x; acc[4 * e + 1] += w * v[e].y; acc[4 * e + 2] += w * v[e].z; acc[4 * e + 3] += w * v[e].w;
+        }
+      }
+      const float inv = 1.f / L;
+      bf16* dst = a.out + m * H * HD + h * HD + d0;
+#pragma unroll
+      for (int e = 0; e < HD / 8; ++e) {
+        uint2 pk;
+        pk.x = pack_bf16(acc[4 * e] * inv, acc[4 * e + 1] * inv);
+        pk.y = pack_bf16(acc[4 * e + 2] * inv, acc[4 * e + 3] * inv);
+        *reinterpret_cast<uint2*>(dst + e * 4) = pk;
+      }
+    }
+  }
 }
 
 }  // namespace spec

@@ -182,7 +182,7 @@ struct spec_ctx {
   int gemm_ctas = SM_SLOTS;            // persistent CTAs of the weight-streaming GEMM
   int l2_prefetch = 0;                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
   std::vector<int> h_parent, h_depth, h_rank;
-  std::vector<int> n_hi;               // host upper bound of committed lengths
+  std::vector<int> n_hi, n_lo;         // host upper / lower bounds of the committed lengths
   std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, mw, mb;
   std::vector<const float*> an, fn;
   const void *embed, *lm_head;
@@ -203,6 +203,7 @@ struct spec_ctx {
   // optional device timeline of the last step: four stamps per launch (see KTrace)
   bool trace_on = false;
   unsigned long long* d_trace = nullptr;
+  unsigned int* d_attn_arrive = nullptr;
   int trace_n = 0;
   std::vector<std::string> trace_names;
   std::vector<unsigned long long> trace_init;
@@ -287,13 +288,14 @@ size_t carve(spec_ctx* c, void* base) {
   c->ntile_lm = c->tc ? ((V + 127) / 128) * 4 : 1;   // argmax partials per row (tile x lane quarter)
   c->topk_slice = (V + SM_SLOTS - 1) / SM_SLOTS;
   c->topk_blocks = (V + c->topk_slice - 1) / c->topk_slice;
-  c->nsplit_attn = c->tc ? (SM_SLOTS / (f.n_heads * B) < 1 ? 1 : (SM_SLOTS / (f.n_heads * B) > 16 ? 16 : SM_SLOTS / (f.n_heads * B))) : 1;
+  c->nsplit_attn = c->tc ? std::max(1, std::min(16, (SM_SLOTS / 2) / (f.n_heads * B))) : 1;   // most KV splits a launch may use
   int Mlog = (int)round_up((size_t)B * T, 16);
   c->keep_logits = !c->tc || (f.flags & SPEC_FLAG_KEEP_LOGITS) || f.accept_mode == 1;
   size_t M = c->Mcap;
 
   c->d_status = b.take<int>(4);
   c->d_trace = b.take<unsigned long long>((size_t)TRACE_CAP * 4);
+  c->d_attn_arrive = b.take<unsigned int>((size_t)B * f.n_heads);
   c->d_n = b.take<int>(B); c->d_cnt = b.take<int>(B); c->d_n_old = b.take<int>(B); c->d_root = b.take<int>(B);
   c->d_count = b.take<int>(B); c->d_path = b.take<int>((size_t)B * (K + 1)); c->d_out_tok = b.take<int>((size_t)B * (K + 1));
   c->d_gen_cnt = b.take<int>(B); c->d_gen_log = b.take<int>((size_t)B * c->gen_cap);
@@ -443,43 +445,54 @@ int linear_simple(spec_ctx* c, const T* x, int ldx, const T* W, float* y, int ld
     if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string(name) + ": " + cudaGetErrorString(e_)); \
   } while (0)
 
-int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l) {
+// n_hi_pass / n_lo_pass: host bounds of the cached length the pass's rows sit on, per sequence
+// (n_lo_pass may be null: nothing is fetched before the dependency wait).
+int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* n_hi_pass, const int* n_lo_pass) {
   const spec_config& f = c->cfg;
-  int H = f.n_heads, D = f.head_dim, HD = H * D, M = c->B * R;
+  int H = f.n_heads, D = f.head_dim;
   AttnTcArgs a{};
   a.q = static_cast<const bf16*>(c->d_q); a.part_o = c->d_part_o; a.part_ml = c->d_part_ml;
   a.pool = static_cast<const bf16*>(c->d_pool); a.g = c->geom; a.page_table = c->d_page_table; a.rows = rows;
-  a.layer = l; a.H = H; a.nsplit = c->nsplit_attn; a.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+  a.layer = l; a.H = H; a.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+  a.out = static_cast<bf16*>(c->d_attn); a.arrive = c->d_attn_arrive;
   a.status = c->d_status;
-  dim3 grid(H, c->nsplit_attn, c->B);
+  int tiles_hi = 1;
+  for (int b = 0; b < c->B; ++b) {
+    tiles_hi = std::max(tiles_hi, (n_hi_pass[b] + R + 63) / 64);
+    if (b < ATTN_MAX_SEQS) a.n_lo[b] = n_lo_pass ? n_lo_pass[b] : 0;
+  }
+  // short contexts: one CTA per (sequence, head) walks all tiles (no merge step); longer ones are cut
+  // into at most one split per resident CTA slot, eight tiles or more each
+  const int slots1 = std::max(1, std::min(c->nsplit_attn, (SM_SLOTS / 2) / (H * c->B)));
+  a.nsplit = tiles_hi <= 12 ? 1 : std::min(slots1, (tiles_hi + 7) / 8);
+  a.stages = ATTN_MAX_STAGES;
+  a.tps = (tiles_hi + a.nsplit - 1) / a.nsplit;
+  dim3 grid(H, a.nsplit, c->B);
   int nw = (R + 15) / 16;
-  size_t rowb = (size_t)D * 2;
-#define ATTN_CASE(HDV, NWV)                                                                              \
+#define ATTN_CASE(HDV, NWV, KGV)                                                                         \
   {                                                                                                    \
-    size_t sm = (size_t)NWV * 16 * rowb + 4 * 64 * rowb + 64;                                          \
+    size_t sm = attention_tc_smem(HDV, NWV, a.stages);                                                 \
     static bool set_ = false;                                                                          \
-    if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_tc<HDV, NWV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); set_ = true; } \
-    KLAUNCH("attention_tc", (attention_tc<HDV, NWV>), grid, dim3(NWV * 32), sm, a);                    \
+    if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_tc<HDV, NWV, KGV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_tc_smem(HDV, NWV, ATTN_MAX_STAGES))); set_ = true; } \
+    KLAUNCH("attention_tc", (attention_tc<HDV, NWV, KGV>), grid, dim3(NWV * KGV * 32), sm, a);         \
   }
   {
+    // up to 64 rows: two key groups of warps per CTA; more rows: one
     ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
     if (D == 128) {
-      if (nw <= 1) ATTN_CASE(128, 1) else if (nw <= 2) ATTN_CASE(128, 2) else if (nw <= 4) ATTN_CASE(128, 4) else ATTN_CASE(128, 8)
+      if (nw <= 1) ATTN_CASE(128, 1, 2) else if (nw <= 2) ATTN_CASE(128, 2, 2) else if (nw <= 4) ATTN_CASE(128, 4, 2) else ATTN_CASE(128, 8, 1)
     } else {
-      if (nw <= 1) ATTN_CASE(64, 1) else if (nw <= 2) ATTN_CASE(64, 2) else if (nw <= 4) ATTN_CASE(64, 4) else ATTN_CASE(64, 8)
+      if (nw <= 1) ATTN_CASE(64, 1, 2) else if (nw <= 2) ATTN_CASE(64, 2, 2) else if (nw <= 4) ATTN_CASE(64, 4, 2) else ATTN_CASE(64, 8, 1)
     }
   }
 #undef ATTN_CASE
-  size_t total = (size_t)M * HD / 4;
-  KLAUNCH("attention_combine", attention_combine, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, c->d_part_o, c->d_part_ml,
-          c->nsplit_attn, rows, H, D, static_cast<bf16*>(c->d_attn));
   return SPEC_OK;
 }
 
 // One pass of the base model over M = B*R rows whose tokens/positions/slots are prepared and
 // whose embeddings are in d_x: bf16 tensor-core path. Leaves the final hidden state in d_hid
 // (float32) and d_hq (bf16).
-int forward_layers_tc(spec_ctx* c, int R, bool chain) {
+int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, const int* n_lo_pass) {
   const spec_config& f = c->cfg;
   Rows rows = make_rows(c, R, chain);
   const int M = c->B * R, d = f.d_model, F = f.d_ffn, H = f.n_heads, D = f.head_dim, HD = H * D, KD = f.n_kv_heads * D;
@@ -501,7 +514,7 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain) {
     }
     KLAUNCH("rope_store_tc", rope_store_tc, dim3(M, M <= 128 ? 4 : 1), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope,
             static_cast<bf16*>(c->d_q), static_cast<bf16*>(c->d_pool), c->geom, c->d_page_table, l, H);
-    if ((r = launch_attention_tc(c, rows, R, l))) return r;
+    if ((r = launch_attention_tc(c, rows, R, l, n_hi_pass, n_lo_pass))) return r;
     PartView vo{};
     {
       const void* mats[1] = {c->wo[l]};
@@ -533,8 +546,8 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain) {
 
 // The same pass with the plain CUDA-core kernels (float32 configurations and the bf16 debug mode).
 template <typename T>
-int forward_layers(spec_ctx* c, int R, bool chain) {
-  if (c->tc) return forward_layers_tc(c, R, chain);
+int forward_layers(spec_ctx* c, int R, bool chain, const int* n_hi_pass, const int* n_lo_pass) {
+  if (c->tc) return forward_layers_tc(c, R, chain, n_hi_pass, n_lo_pass);
   const spec_config& f = c->cfg;
   Rows rows = make_rows(c, R, chain);
   int M = c->B * R, d = f.d_model, F = f.d_ffn, H = f.n_heads, D = f.head_dim, HD = H * D;
@@ -661,7 +674,9 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
     prepare_prefill_rows<T><<<M, 128, 0, c->stream>>>(rows, c->d_prompt, c->d_offsets, ch, static_cast<const T*>(c->embed), c->d_x,
                                                     f.d_model, f.vocab, c->d_status);
     LAUNCH_CHECK("prepare_prefill_rows");
-    int r = forward_layers<T>(c, R, true);
+    std::vector<int> n_pass(batch);
+    for (int b = 0; b < batch; ++b) n_pass[b] = std::min(offsets[b + 1] - offsets[b], ch * R);
+    int r = forward_layers<T>(c, R, true, n_pass.data(), nullptr);
     if (r) return r;
     prefill_keep_last<T><<<batch, 256, 0, c->stream>>>(rows, c->d_offsets, ch, c->d_hid, c->d_h_last, static_cast<T*>(c->d_hq_last), f.d_model);
     LAUNCH_CHECK("prefill_keep_last");
@@ -674,6 +689,7 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
   if (r) return r;
   c->n_hi.assign(batch, 0);
   for (int b = 0; b < batch; ++b) c->n_hi[b] = offsets[b + 1] - offsets[b];
+  c->n_lo = c->n_hi;
   c->prefilled = true;
   return SPEC_OK;
 }
@@ -724,7 +740,7 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
           (const int*)c->d_depth, (const int*)c->d_rank, c->cap, static_cast<const T*>(c->embed), c->d_x, d, f.vocab, c->d_status);
   cudaEventRecord(c->phase_ev[2], c->stream);
   // (3) verification forward
-  int r = forward_layers<T>(c, T_, false);
+  int r = forward_layers<T>(c, T_, false, c->n_hi.data(), c->n_lo.data());
   if (r) return r;
   r = lm_head_argmax<T>(c, static_cast<const T*>(c->d_hq), M);
   if (r) return r;
@@ -759,9 +775,9 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     CUDA_OK(cudaMemcpyAsync(nn.data(), c->d_n, B * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
     r = check_status(c);   // synchronises
     if (r) return r;
-    for (int b = 0; b < B; ++b) c->n_hi[b] = nn[b];
+    for (int b = 0; b < B; ++b) c->n_hi[b] = c->n_lo[b] = nn[b];
   } else {
-    for (int b = 0; b < B; ++b) c->n_hi[b] += K + 1;
+    for (int b = 0; b < B; ++b) { c->n_hi[b] += K + 1; c->n_lo[b] += 1; }
   }
   return SPEC_OK;
 }
@@ -856,6 +872,7 @@ int spec_create(const spec_config* cfg, const spec_weights* w, const spec_tree* 
   up(c->d_mw, c->mw.data(), c->mw.size() * sizeof(void*));
   up(c->d_mb, c->mb.data(), c->mb.size() * sizeof(void*));
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 4 * sizeof(int), c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_attn_arrive, 0, (size_t)cfg->max_batch * cfg->n_heads * sizeof(unsigned int), c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_cand, 0, (size_t)cfg->max_batch * (c->K + 1) * c->kmax * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) { g_create_error = std::string("set-up copies: ") + cudaGetErrorString(e); delete c; return SPEC_E_CUDA; }
@@ -896,7 +913,7 @@ int spec_read_generated(spec_ctx* c, int32_t seq, int32_t* out, int32_t max_toke
   std::vector<int> nn(c->B);
   CUDA_OK(cudaMemcpyAsync(nn.data(), c->d_n, c->B * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(cudaStreamSynchronize(c->stream));
-  for (int b = 0; b < c->B; ++b) c->n_hi[b] = nn[b];
+  for (int b = 0; b < c->B; ++b) c->n_hi[b] = c->n_lo[b] = nn[b];
   return SPEC_OK;
 }
 
