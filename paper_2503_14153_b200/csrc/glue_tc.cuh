@@ -193,6 +193,94 @@ swiglu_reduce_tc(const PartView pv, int gp0, int up0, bf16* __restrict__ act, in
   }
 }
 
+// ------------------------------------------------------------------ extra decoding heads
+// r[b*K + k0 + kk][i] = bf16(h + SiLU(z + bias_k[i])), z = sum of the partial slots of head
+// matrix kk of this launch group (padded columns kk * dpad + i), h = hq_last[b][i] (already
+// bf16). grid (B * nk, CTAs per row).
+__global__ void __launch_bounds__(256)
+medusa_act_tc(const PartView pv, int dpad, const bf16* __restrict__ hq_last, const bf16* const* __restrict__ bias,
+              bf16* __restrict__ r, int K, int k0, int nk, int d, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  const int b = blockIdx.x / nk, kk = blockIdx.x % nk, k = k0 + kk;
+  const bf16* bk = bias[k];
+  for (int c4 = blockIdx.y * blockDim.x + threadIdx.x; c4 < (d >> 2); c4 += gridDim.y * blockDim.x) {
+    const int i = c4 * 4;
+    const float4 z = part_sum4(pv, b, kk * dpad + i);
+    const uint2 hraw = *reinterpret_cast<const uint2*>(hq_last + (size_t)b * d + i);
+    const uint2 braw = *reinterpret_cast<const uint2*>(bk + i);
+    const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hraw);
+    const __nv_bfloat162* bp = reinterpret_cast<const __nv_bfloat162*>(&braw);
+    const float2 h01 = __bfloat1622float2(hp[0]), h23 = __bfloat1622float2(hp[1]);
+    const float2 b01 = __bfloat1622float2(bp[0]), b23 = __bfloat1622float2(bp[1]);
+    *reinterpret_cast<uint2*>(r + ((size_t)b * K + k) * d + i) =
+        pack4_bf16(h01.x + silu_f(z.x + b01.x), h01.y + silu_f(z.y + b01.y), h23.x + silu_f(z.z + b23.x), h23.y + silu_f(z.w + b23.y));
+  }
+}
+
+// Each row's kmax best (value desc, index asc) of this block's slice of the logits go to the
+// partial lists pk_val / pk_idx [block][rows][kmax]. grid (slices, rows); dynamic shared
+// memory: slice floats.
+__global__ void __launch_bounds__(256)
+topk_slices(const float* __restrict__ logits, int V, int rows_total, int slice, int kmax, float* __restrict__ pk_val,
+            int* __restrict__ pk_idx, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  extern __shared__ float zs[];
+  const int row = blockIdx.y, n0 = blockIdx.x * slice, n1 = min(n0 + slice, V);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  for (int c = threadIdx.x; c < n1 - n0; c += blockDim.x) zs[c] = logits[(size_t)row * V + n0 + c];
+  __syncthreads();
+  __shared__ float sv[8];
+  __shared__ int si[8];
+  for (int t = 0; t < kmax; ++t) {
+    float bv = -INFINITY; int bi = 0x7fffffff;
+    for (int c = threadIdx.x; c < n1 - n0; c += blockDim.x) if (better(zs[c], n0 + c, bv, bi)) { bv = zs[c]; bi = n0 + c; }
+    warp_argmax(bv, bi);
+    if (lane == 0) { sv[warp] = bv; si[warp] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 1; w < nw; ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
+      const size_t o = ((size_t)blockIdx.x * rows_total + row) * kmax + t;
+      pk_val[o] = bv;
+      pk_idx[o] = bi;
+      if (bi != 0x7fffffff) zs[bi - n0] = -INFINITY;
+    }
+    __syncthreads();
+  }
+}
+
+// Finishes the per-row argmax from the per-(tile, lane quarter) partials of the lm_head
+// epilogue: one CTA per row, result in pval2[m] / pidx2[m].
+__global__ void __launch_bounds__(256)
+argmax_finish(const float* __restrict__ pval, const int* __restrict__ pidx, int ntile, float* __restrict__ pval2,
+              int* __restrict__ pidx2, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  const int m = blockIdx.x;
+  float bv = -INFINITY; int bi = 0x7fffffff;
+  for (int t = threadIdx.x; t < ntile; t += blockDim.x) {
+    const float v = pval[(size_t)m * ntile + t]; const int i = pidx[(size_t)m * ntile + t];
+    if (better(v, i, bv, bi)) { bv = v; bi = i; }
+  }
+  __shared__ float sv[8];
+  __shared__ int si[8];
+  warp_argmax(bv, bi);
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
+    pval2[m] = bv;
+    pidx2[m] = bi;
+  }
+}
+
 // y[m][n] = sum of the partial slots (logical columns of a single matrix): the stand-alone linear.
 __global__ void __launch_bounds__(256)
 part_sum_rows(const PartView pv, float* __restrict__ y, int M, int N) {

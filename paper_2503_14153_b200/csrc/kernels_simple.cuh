@@ -33,7 +33,19 @@ __global__ void prepare_verify_rows(Rows rows, const int* __restrict__ cand, int
     if (i == 0) rows.cnt[b] = ok ? rows.R : 0;
   }
   const T* e = embed + (size_t)t * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)m * d + c] = to_f<T>(e[c]);
+  if (sizeof(T) == 2 && d % 8 == 0) {
+    // 16-byte loads of the embedding row, all in flight at once
+    for (int c8 = threadIdx.x; c8 < (d >> 3); c8 += blockDim.x) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(e) + c8 * 8);
+      const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&raw);
+      const float2 f0 = __bfloat1622float2(hp[0]), f1 = __bfloat1622float2(hp[1]), f2 = __bfloat1622float2(hp[2]), f3 = __bfloat1622float2(hp[3]);
+      float* dst = x + (size_t)m * d + c8 * 8;
+      *reinterpret_cast<float4*>(dst) = make_float4(f0.x, f0.y, f1.x, f1.y);
+      *reinterpret_cast<float4*>(dst + 4) = make_float4(f2.x, f2.y, f3.x, f3.y);
+    }
+  } else {
+    for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)m * d + c] = to_f<T>(e[c]);
+  }
 }
 
 // Prefill pass number `chunk`: row i of sequence b is prompt token chunk*R + i.
@@ -370,6 +382,7 @@ struct AcceptArgs {
   const float* hid;            // [rows][d]
   int *am, *path, *count, *out_tok, *n_old, *root_tok;
   float* h_last;
+  bf16* hq_last;               // optional bf16 copy of h_last (operand of the extra heads' GEMM)
   int *gen_log, *gen_cnt, gen_cap;
 };
 
@@ -464,7 +477,11 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptArgs a, unsigned long
   __syncthreads();
   if (len_s > 0) {
     const float* src = a.hid + (size_t)(m0 + last_s) * a.d;
-    for (int c = threadIdx.x; c < a.d; c += blockDim.x) a.h_last[(size_t)b * a.d + c] = src[c];
+    for (int c = threadIdx.x; c < a.d; c += blockDim.x) {
+      const float v = src[c];
+      a.h_last[(size_t)b * a.d + c] = v;
+      if (a.hq_last) a.hq_last[(size_t)b * a.d + c] = __float2bfloat16_rn(v);
+    }
   }
 }
 

@@ -204,6 +204,9 @@ struct spec_ctx {
   bool trace_on = false;
   unsigned long long* d_trace = nullptr;
   unsigned int* d_attn_arrive = nullptr;
+  float* d_pval2 = nullptr;            // finished per-row argmax (tensor-core path)
+  int* d_pidx2 = nullptr;
+  float* d_head_logits = nullptr;      // [B*K][vocab] logits of the extra heads (tensor-core path)
   int trace_n = 0;
   std::vector<std::string> trace_names;
   std::vector<unsigned long long> trace_init;
@@ -296,6 +299,8 @@ size_t carve(spec_ctx* c, void* base) {
   c->d_status = b.take<int>(4);
   c->d_trace = b.take<unsigned long long>((size_t)TRACE_CAP * 4);
   c->d_attn_arrive = b.take<unsigned int>((size_t)B * f.n_heads);
+  c->d_pval2 = b.take<float>(c->Mcap); c->d_pidx2 = b.take<int>(c->Mcap);
+  c->d_head_logits = c->tc ? b.take<float>(round_up((size_t)B * (K ? K : 1), 16) * V, 1024) : nullptr;
   c->d_n = b.take<int>(B); c->d_cnt = b.take<int>(B); c->d_n_old = b.take<int>(B); c->d_root = b.take<int>(B);
   c->d_count = b.take<int>(B); c->d_path = b.take<int>((size_t)B * (K + 1)); c->d_out_tok = b.take<int>((size_t)B * (K + 1));
   c->d_gen_cnt = b.take<int>(B); c->d_gen_log = b.take<int>((size_t)B * c->gen_cap);
@@ -340,7 +345,7 @@ size_t carve(spec_ctx* c, void* base) {
   c->d_u = b.take<uint8_t>(M * d * e, 1024); c->d_q = b.take<uint8_t>(M * HD * e, 1024);
   c->d_attn = b.take<uint8_t>(M * HD * e, 1024); c->d_act = b.take<uint8_t>(M * F * e, 1024);
   c->d_hq = b.take<uint8_t>(M * d * e, 1024); c->d_hq_last = b.take<uint8_t>(round_up((size_t)B, 16) * d * e, 1024);
-  c->d_r = b.take<uint8_t>((size_t)B * (K ? K : 1) * d * e, 1024);
+  c->d_r = b.take<uint8_t>(round_up((size_t)B * (K ? K : 1), 16) * d * e, 1024);
   c->geom = KVGeom{f.n_layers, f.n_kv_heads, f.head_dim, f.page_size, c->pages_per_seq, B};
   size_t pool_elems = (size_t)B * c->pages_per_seq * c->geom.page_elems();
   c->d_pool = b.take<uint8_t>(pool_elems * e, 1024);
@@ -593,27 +598,65 @@ int forward_layers(spec_ctx* c, int R, bool chain, const int* n_hi_pass, const i
   return SPEC_OK;
 }
 
+// lm_head on the tensor cores over `M` bf16 operand rows at `src`: each CTA owns whole weight
+// tiles, leaves per-(row, tile, lane quarter) argmax partials and, if asked, the logits.
+int lm_head_gemm_tc(spec_ctx* c, const void* src, int M, float* logits) {
+  const spec_config& f = c->cfg;
+  GemmPlan g;
+  int rws[1] = {f.vocab};
+  if (!plan_gemm(M, f.d_model, 1, rws, c->gemm_ctas, true, &g)) return c->fail(SPEC_E_BADARG, "unsupported lm_head shape");
+  StreamTmaps tm{};
+  const CUtensorMap* ta = c->tmap(c->lm_head, f.vocab, f.d_model, 128);
+  const CUtensorMap* tb = c->tmap(src, std::max<size_t>(round_up(M, 16), g.MT), f.d_model, g.MT);
+  if (!ta || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
+  tm.a[0] = *ta; tm.b = *tb;
+  g.p.logits = logits; g.p.ld_logits = f.vocab;
+  g.p.pval = c->d_pval; g.p.pidx = c->d_pidx;
+  g.p.l2_prefetch = c->l2_prefetch;
+  g.p.status = c->d_status;
+  g.p.trace = c->next_trace("gemm_lm_head");
+  cudaError_t e = launch_gs(c->stream, c->pdl, g, tm);
+  c->launches++;
+  if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_stream lm_head launch: ") + cudaGetErrorString(e));
+  return SPEC_OK;
+}
+
+// Extra decoding heads on the tensor cores: residual blocks (head matrices stacked along the
+// output dimension, up to four per launch), shared lm_head, per-head top-k.
+int heads_tc(spec_ctx* c, const int* ov) {
+  const spec_config& f = c->cfg;
+  const int B = c->B, K = c->K, d = f.d_model, kmax = c->kmax, rows_total = B * K;
+  const int dpad = (d + 127) / 128 * 128;
+  for (int k0 = 0; k0 < K; k0 += GS_MAX_MATS) {
+    const int nk = std::min(GS_MAX_MATS, K - k0);
+    const void* mats[GS_MAX_MATS];
+    int rws[GS_MAX_MATS];
+    for (int i = 0; i < nk; ++i) { mats[i] = c->mw[k0 + i]; rws[i] = d; }
+    PartView pv{};
+    int r = run_gemm(c, c->d_hq_last, B, d, nk, mats, rws, SPEC_PROFILE_OFF, &pv);
+    if (r) return r;
+    KLAUNCH("medusa_act_tc", medusa_act_tc, dim3(B * nk, 4), dim3(256), 0, pv, dpad, (const bf16*)c->d_hq_last,
+            reinterpret_cast<const bf16* const*>(c->d_mb), static_cast<bf16*>(c->d_r), K, k0, nk, d);
+  }
+  int r = lm_head_gemm_tc(c, c->d_r, rows_total, c->d_head_logits);
+  if (r) return r;
+  KLAUNCH("topk_slices", topk_slices, dim3(c->topk_blocks, rows_total), dim3(256), (size_t)c->topk_slice * sizeof(float),
+          (const float*)c->d_head_logits, f.vocab, rows_total, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
+  size_t sm2 = (size_t)c->topk_blocks * kmax * 8;
+  KLAUNCH("topk_merge", topk_merge, dim3(rows_total), dim3(256), sm2, (const float*)c->d_pk_val, (const int*)c->d_pk_idx,
+          c->topk_blocks, rows_total, K, kmax, (const int*)c->d_root, ov, c->d_cand);
+  return SPEC_OK;
+}
+
 // lm_head over `M` operand rows at `src`, leaving per-row argmax partials (and logits).
 template <typename T>
 int lm_head_argmax(spec_ctx* c, const T* src, int M) {
   const spec_config& f = c->cfg;
   if (c->tc) {
-    GemmPlan g;
-    int rws[1] = {f.vocab};
-    if (!plan_gemm(M, f.d_model, 1, rws, c->gemm_ctas, true, &g)) return c->fail(SPEC_E_BADARG, "unsupported lm_head shape");
-    StreamTmaps tm{};
-    const CUtensorMap* ta = c->tmap(c->lm_head, f.vocab, f.d_model, 128);
-    const CUtensorMap* tb = c->tmap(src, std::max<size_t>(round_up(M, 16), g.MT), f.d_model, g.MT);
-    if (!ta || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
-    tm.a[0] = *ta; tm.b = *tb;
-    g.p.logits = c->keep_logits ? c->d_logits : nullptr; g.p.ld_logits = f.vocab;
-    g.p.pval = c->d_pval; g.p.pidx = c->d_pidx;
-    g.p.l2_prefetch = c->l2_prefetch;
-    g.p.status = c->d_status;
-    g.p.trace = c->next_trace("gemm_lm_head");
-    cudaError_t e = launch_gs(c->stream, c->pdl, g, tm);
-    c->launches++;
-    if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_stream lm_head launch: ") + cudaGetErrorString(e));
+    int r = lm_head_gemm_tc(c, src, M, c->keep_logits ? c->d_logits : nullptr);
+    if (r) return r;
+    KLAUNCH("argmax_finish", argmax_finish, dim3(M), dim3(256), 0, (const float*)c->d_pval, (const int*)c->d_pidx, c->ntile_lm,
+            c->d_pval2, c->d_pidx2);
   } else {
     int r = linear_simple<T>(c, src, f.d_model, static_cast<const T*>(c->lm_head), c->d_logits, f.vocab, M, f.vocab, f.d_model);
     if (r) return r;
@@ -626,7 +669,8 @@ int lm_head_argmax(spec_ctx* c, const T* src, int M) {
 AcceptArgs make_accept(spec_ctx* c, int R, int mode) {
   AcceptArgs a{};
   a.rows = make_rows(c, R, false);
-  a.pval = c->d_pval; a.pidx = c->d_pidx; a.ntile = c->ntile_lm;
+  a.pval = c->tc ? c->d_pval2 : c->d_pval; a.pidx = c->tc ? c->d_pidx2 : c->d_pidx; a.ntile = 1;
+  a.hq_last = c->tc ? static_cast<bf16*>(c->d_hq_last) : nullptr;
   a.parent = c->d_parent; a.depth = c->d_depth; a.edge_ok = nullptr;
   a.K = c->K; a.frag_token = c->cfg.frag_token; a.d = c->cfg.d_model; a.mode = mode;
   a.hid = c->d_hid; a.am = c->d_am; a.path = c->d_path; a.count = c->d_count; a.out_tok = c->d_out_tok;
@@ -715,7 +759,10 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     ov = c->d_cand_ov;
   }
   // (1) extra heads -> shared lm_head -> per-head top-k -> candidate table
-  if (K > 0) {
+  if (K > 0 && c->tc) {
+    int r = heads_tc(c, ov);
+    if (r) return r;
+  } else if (K > 0) {
     constexpr int MC = 4;
     dim3 g1((K * d + 7) / 8, (B + MC - 1) / MC);
     KLAUNCH("medusa_resblock", (medusa_resblock<T, MC>), g1, dim3(256), 0, (const float*)c->d_h_last,
