@@ -147,12 +147,13 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
     if (lane == 0) {
       // ---- TMA producer ----
       const int n_units = hi - lo;
+      const uint64_t wpol = l2_policy_evict_first();
       const int n_pre = n_units < STAGES ? n_units : STAGES;
       // weights first: they do not depend on the kernel before this one
       for (int i = 0; i < n_pre; ++i) {
         GsUnit w = gs_decode(p, lo + i);
         mbar_expect_tx(&full[i], Cfg::STAGE_BYTES);
-        tma_load_2d(tiles + i * Cfg::STAGE_BYTES, &tm.a[w.mat], w.kc * Cfg::BK, w.row0, &full[i]);
+        tma_load_2d_hint(tiles + i * Cfg::STAGE_BYTES, &tm.a[w.mat], w.kc * Cfg::BK, w.row0, &full[i], wpol);
       }
       {
         int n_pf = n_units - n_pre;
@@ -176,7 +177,7 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
         GsUnit w = gs_decode(p, lo + issued);
         uint8_t* a = tiles + st * Cfg::STAGE_BYTES;
         mbar_expect_tx(&full[st], Cfg::STAGE_BYTES);
-        tma_load_2d(a, &tm.a[w.mat], w.kc * Cfg::BK, w.row0, &full[st]);
+        tma_load_2d_hint(a, &tm.a[w.mat], w.kc * Cfg::BK, w.row0, &full[st], wpol);
         tma_load_2d(a + Cfg::A_BYTES, &tm.b, w.kc * Cfg::BK, w.mt * MT, &full[st]);
       }
       if (!ok) {
