@@ -313,7 +313,7 @@ def main():
         dec.profile_kernel(B.PROFILE_OFF)
         if k_n > 0:
             per = k_ms / k_n * 1e-3
-            out["roofline"] = {"bound": "hbm", "kernel": "gemm_tc<64,SWIGLU> (gate+up projection, fused SwiGLU)",
+            out["roofline"] = {"bound": "hbm", "kernel": "gemm_stream<64> on the gate+up projection (2 x [11008,4096] bf16 weights streamed once)",
                                "achieved": gate_up_b / per / 1e9, "peak": peak, "unit": "GB/s",
                                "frac": gate_up_b / per / 1e9 / peak, "traffic": None, "peak_kind": peak_kind,
                                "launches_timed": int(k_n), "us_per_launch": per * 1e6,
@@ -328,6 +328,23 @@ def main():
             per_kernel[name] = k_ms / max(k_n, 1) * 1e3
         dec.profile_kernel(B.PROFILE_OFF)
         out["kernel_us"] = per_kernel
+        # device timeline of one step (GPU global timer): per kernel kind, span from first block start to
+        # last block end, averaged over its launches; the GEMMs also report operands-landed -> last MMA issued
+        dec.set_option(B.OPT_TRACE, 1)
+        dec.step_async()
+        tr = dec.trace()
+        dec.set_option(B.OPT_TRACE, 0)
+        agg = {}
+        for name, t_start, t_end, m2, m3 in tr:
+            a = agg.setdefault(name, [0, 0.0, 0.0])
+            a[0] += 1
+            a[1] += (t_end - t_start) / 1e3
+            if name.startswith("gemm") and m2 < (1 << 62) and m3 > 0:
+                a[2] += (m3 - m2) / 1e3
+        out["timeline_us"] = {k: {"launches": v[0], "span_avg": round(v[1] / v[0], 2),
+                                  **({"stream_window_avg": round(v[2] / v[0], 2)} if v[2] > 0 else {})} for k, v in agg.items()}
+        if tr:
+            out["timeline_us"]["step_span"] = round((max(r[2] for r in tr) - min(r[1] for r in tr)) / 1e3, 1)
 
     if want_cpu:
         dt, cnt, threads = oracle_step_sample(cfg, host_w, tree)
