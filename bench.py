@@ -315,7 +315,11 @@ def main():
             per = k_ms / k_n * 1e-3
             out["roofline"] = {"bound": "hbm", "kernel": "gemm_stream<64> on the gate+up projection (2 x [11008,4096] bf16 weights streamed once)",
                                "achieved": gate_up_b / per / 1e9, "peak": peak, "unit": "GB/s",
-                               "frac": gate_up_b / per / 1e9 / peak, "traffic": None, "peak_kind": peak_kind,
+                               "frac": gate_up_b / per / 1e9 / peak,
+                               # dram__bytes_read.sum + dram__bytes_write.sum of this kernel at this shape
+                               # (profiles/gemm_stream_7b_shapes_ncu_full.md); null for other shapes
+                               "traffic": 189.9e6 if (cfg.d_model, cfg.d_ffn, T) == (4096, 11008, 64) else None,
+                               "peak_kind": peak_kind,
                                "launches_timed": int(k_n), "us_per_launch": per * 1e6,
                                "algorithmic_bytes_per_launch": gate_up_b}
         per_kernel = {}
