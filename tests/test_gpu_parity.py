@@ -81,6 +81,13 @@ def test_small_bf16_d128_tree64_tensor_core_path(torch):
     assert rep.max_logit_err < TOL_BF16
 
 
+def test_ten_heads_deep_tree(torch):
+    """The paper's head count (K = 10): ten stacked head matrices (three GEMM launches), a tree ten levels deep."""
+    cfg = SMALL_BF16.with_(name="small_bf16_k10", n_medusa=10, topk=(4, 3, 2, 2, 2, 1, 1, 1, 1, 1), tree_nodes=48, seed=23)
+    rep = _lockstep(cfg, TOL_BF16, 16, prompt_len=40)
+    assert rep.max_logit_err < TOL_BF16
+
+
 def test_controlled_draft_accept_lengths(torch):
     """Controlled-acceptance draft: rank-0 candidate of head j is the true greedy token with
     probability p. The stream is unchanged and the accepted lengths match the oracle's."""
