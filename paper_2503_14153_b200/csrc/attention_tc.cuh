@@ -136,12 +136,26 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   }
   pdl_wait();
   if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  // sequence state, ancestor sets and the Q tile are independent loads: one trip for all of them
   const int R = a.rows.R, cnt = a.rows.cnt[b], n = a.rows.n[b];
+  const int i0 = rg * 16 + (lane >> 2), i1 = i0 + 8;        // this thread's two query rows
+  uint32_t anc0[4], anc1[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) { anc0[w] = a.rows.anc[i0 * 4 + w]; anc1[w] = a.rows.anc[i1 * 4 + w]; }
+  constexpr int QC = NW * 16 * (HD / 8);                      // 16-byte chunks of the Q tile
+  constexpr int PER = (QC + NTHR - 1) / NTHR;
+  uint4 qv[PER];
+#pragma unroll
+  for (int k = 0; k < PER; ++k) {
+    const int c = threadIdx.x + k * NTHR;
+    const int r = c / (HD / 8), ch = c % (HD / 8);
+    qv[k] = make_uint4(0, 0, 0, 0);
+    if (c < QC && r < R) qv[k] = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + r) * H * HD + h * HD + ch * 8);
+  }
   const int S = n + cnt;
   const int M = a.rows.B * R;
   const int total_tiles = (S + KT - 1) / KT;
   const int t1 = min(total_tiles, t0 + tps);
-  const int i0 = rg * 16 + (lane >> 2), i1 = i0 + 8;        // this thread's two query rows
   if (cnt == 0) {
     // inactive sequence: let the copies already in flight land before the CTA goes away
     if (threadIdx.x == 0)
@@ -151,27 +165,14 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   // the rest of the first tiles
   if (threadIdx.x == 0)
     for (int i = pre; i < ST && t0 + i < t1; ++i) issue(t0 + i, i);
-  // ancestor sets and Q (rows beyond cnt are zero): all loads first, then the swizzled stores
-  uint32_t anc0[4] = {0, 0, 0, 0}, anc1[4] = {0, 0, 0, 0};
-  if (i0 < cnt) for (int w = 0; w < 4; ++w) anc0[w] = a.rows.anc[i0 * 4 + w];
-  if (i1 < cnt) for (int w = 0; w < 4; ++w) anc1[w] = a.rows.anc[i1 * 4 + w];
-  {
-    constexpr int QC = NW * 16 * (HD / 8);                    // 16-byte chunks of the Q tile
-    constexpr int PER = (QC + NTHR - 1) / NTHR;
-    uint4 qv[PER];
+  // rows beyond cnt see nothing and hold zeros
+  if (i0 >= cnt) anc0[0] = anc0[1] = anc0[2] = anc0[3] = 0u;
+  if (i1 >= cnt) anc1[0] = anc1[1] = anc1[2] = anc1[3] = 0u;
 #pragma unroll
-    for (int k = 0; k < PER; ++k) {
-      const int c = threadIdx.x + k * NTHR;
-      const int r = c / (HD / 8), ch = c % (HD / 8);
-      qv[k] = make_uint4(0, 0, 0, 0);
-      if (c < QC && r < cnt) qv[k] = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + r) * H * HD + h * HD + ch * 8);
-    }
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-      const int c = threadIdx.x + k * NTHR;
-      const int r = c / (HD / 8), ch = c % (HD / 8);
-      if (c < QC) *reinterpret_cast<uint4*>(qs + r * ROWB + ((ch ^ (r & 7)) << 4)) = qv[k];
-    }
+  for (int k = 0; k < PER; ++k) {
+    const int c = threadIdx.x + k * NTHR;
+    const int r = c / (HD / 8), ch = c % (HD / 8);
+    if (c < QC) *reinterpret_cast<uint4*>(qs + r * ROWB + ((ch ^ (r & 7)) << 4)) = (r < cnt) ? qv[k] : make_uint4(0, 0, 0, 0);
   }
   __syncthreads();
 

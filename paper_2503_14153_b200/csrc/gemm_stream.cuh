@@ -239,14 +239,26 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
         const int slot = c - p.seg.owner(t * KC);
         float* dst = p.part + (size_t)slot * p.slot_stride + (size_t)nt * 128 + q * 32 + lane;
         const size_t ld = (size_t)p.n_tiles * 128;
-#pragma unroll 1
-        for (int col = 0; col < MT; col += 16) {
+        if (MT >= 32) {
+          // all loads of the accumulator are issued before the first store
+          uint32_t r[MT >= 32 ? MT / 32 : 1][32];
+#pragma unroll
+          for (int g = 0; g < MT / 32; ++g) tmem_ld32(taddr + g * 32, r[g]);
+          tmem_ld_wait();
+#pragma unroll
+          for (int g = 0; g < MT / 32; ++g)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int m = m0 + g * 32 + j;
+              if (m < p.M) dst[(size_t)m * ld] = __uint_as_float(r[g][j]);
+            }
+        } else {
           uint32_t r[16];
-          tmem_ld16(taddr + col, r);
+          tmem_ld16(taddr, r);
           tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            const int m = m0 + col + j;
+            const int m = m0 + j;
             if (m < p.M) dst[(size_t)m * ld] = __uint_as_float(r[j]);
           }
         }

@@ -617,6 +617,9 @@ __global__ void medusa_lmhead_topk(const T* __restrict__ r, const T* __restrict_
 
 // Merges the partial lists of one (sequence, head) row into cand[b][k+1][0..kmax) and applies
 // the optional override table; block 0 of each sequence also writes cand[b][0][0] = root.
+// Every slice's list is already ordered (value desc, index asc), so the row's best kmax are
+// found by a tournament over the list heads: one warp, each lane looking after every 32nd list.
+// Dynamic shared memory: nblocks * kmax * 8 + nblocks * 4 bytes.
 __global__ void topk_merge(const float* __restrict__ pk_val, const int* __restrict__ pk_idx, int nblocks,
                            int rows_total, int K, int kmax, const int* __restrict__ root_tok,
                            const int* __restrict__ cand_override, int* __restrict__ cand, unsigned long long* tr) {
@@ -624,46 +627,47 @@ __global__ void topk_merge(const float* __restrict__ pk_val, const int* __restri
   pdl_launch_dependents();
   pdl_wait();
   if (threadIdx.x == 0) trace_mark_min(tr, 2);
-  extern __shared__ float ms[];     // values [nblocks*kmax] then indices
+  extern __shared__ float ms[];     // values [nblocks*kmax], indices [nblocks*kmax], list positions [nblocks]
   int row = blockIdx.x, b = row / K, k = row % K;
   int total = nblocks * kmax;
   float* v = ms;
   int* ix = reinterpret_cast<int*>(ms + total);
+  int* head = ix + total;
   for (int c = threadIdx.x; c < total; c += blockDim.x) {
     int blk = c / kmax, t = c % kmax;
     size_t o = ((size_t)blk * rows_total + row) * kmax + t;
     v[c] = pk_val[o];
     ix[c] = pk_idx[o];
   }
+  for (int c = threadIdx.x; c < nblocks; c += blockDim.x) head[c] = 0;
   __syncthreads();
-  __shared__ float sv[32];
-  __shared__ int si[32], sp[32];
-  int* out = cand + ((size_t)b * (K + 1) + k + 1) * kmax;
-  for (int t = 0; t < kmax; ++t) {
-    float bv = -INFINITY; int bi = 0x7fffffff, bp = -1;
-    for (int c = threadIdx.x; c < total; c += blockDim.x)
-      if (better(v[c], ix[c], bv, bi)) { bv = v[c]; bi = ix[c]; bp = c; }
-    // warp then block reduction carrying the position
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      int oi = __shfl_xor_sync(0xffffffffu, bi, o), op = __shfl_xor_sync(0xffffffffu, bp, o);
-      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bp = op; }
-    }
-    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; sp[threadIdx.x >> 5] = bp; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      for (int w = 1; w < (blockDim.x >> 5); ++w)
-        if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; bp = sp[w]; }
-      int tokv = bi;
-      if (cand_override) {
-        int o = cand_override[((size_t)b * K + k) * kmax + t];
-        if (o >= 0) tokv = o;
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    int* out = cand + ((size_t)b * (K + 1) + k + 1) * kmax;
+    for (int t = 0; t < kmax; ++t) {
+      float bv = -INFINITY; int bi = 0x7fffffff, bl = -1;
+      for (int l = lane; l < nblocks; l += 32) {
+        const int pos = head[l];
+        if (pos < kmax && better(v[l * kmax + pos], ix[l * kmax + pos], bv, bi)) { bv = v[l * kmax + pos]; bi = ix[l * kmax + pos]; bl = l; }
       }
-      out[t] = (tokv == 0x7fffffff) ? 0 : tokv;
-      if (bp >= 0) v[bp] = -INFINITY, ix[bp] = 0x7fffffff;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        int oi = __shfl_xor_sync(0xffffffffu, bi, o), ol = __shfl_xor_sync(0xffffffffu, bl, o);
+        if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bl = ol; }
+      }
+      // every lane now holds the winner; the lane that looks after its list moves that list on
+      if (bl >= 0 && (bl & 31) == lane) head[bl]++;
+      if (lane == 0) {
+        int tokv = bi;
+        if (cand_override) {
+          int o = cand_override[((size_t)b * K + k) * kmax + t];
+          if (o >= 0) tokv = o;
+        }
+        out[t] = (tokv == 0x7fffffff) ? 0 : tokv;
+      }
+      __syncwarp();
     }
-    __syncthreads();
   }
   if (k == 0 && threadIdx.x == 0) cand[(size_t)b * (K + 1) * kmax] = root_tok[b];
 }

@@ -642,7 +642,7 @@ int heads_tc(spec_ctx* c, const int* ov) {
   if (r) return r;
   KLAUNCH("topk_slices", topk_slices, dim3(c->topk_blocks, rows_total), dim3(256), (size_t)c->topk_slice * sizeof(float),
           (const float*)c->d_head_logits, f.vocab, rows_total, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
-  size_t sm2 = (size_t)c->topk_blocks * kmax * 8;
+  size_t sm2 = (size_t)c->topk_blocks * kmax * 8 + (size_t)c->topk_blocks * 4;
   KLAUNCH("topk_merge", topk_merge, dim3(rows_total), dim3(256), sm2, (const float*)c->d_pk_val, (const int*)c->d_pk_idx,
           c->topk_blocks, rows_total, K, kmax, (const int*)c->d_root, ov, c->d_cand);
   return SPEC_OK;
@@ -773,7 +773,7 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     KLAUNCH("medusa_lmhead_topk", (medusa_lmhead_topk<T, MC>), g2, dim3(256), sm, static_cast<const T*>(c->d_r),
             static_cast<const T*>(c->lm_head), rows_total, f.vocab, d, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
     // partial lists of the row chunks are laid out per block over all rows
-    size_t sm2 = (size_t)c->topk_blocks * kmax * 8;
+    size_t sm2 = (size_t)c->topk_blocks * kmax * 8 + (size_t)c->topk_blocks * 4;
     KLAUNCH("topk_merge", topk_merge, dim3(rows_total), dim3(256), sm2, (const float*)c->d_pk_val, (const int*)c->d_pk_idx,
             c->topk_blocks, rows_total, K, kmax, (const int*)c->d_root, ov, c->d_cand);
   } else {
