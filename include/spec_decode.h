@@ -212,6 +212,17 @@ size_t spec_op_linear_scratch_floats(int32_t M, int32_t N, int32_t K, int32_t ct
 int spec_op_linear(int32_t dtype, const void *x, const void *w, float *y, int32_t M, int32_t N,
                    int32_t K, int32_t ctas, float *scratch, void *cuda_stream);
 
+/* Syntax-enriched training labels (Sec. III-C). tokens: DEVICE int32 [n_seq][seq_len], each row
+ * the token ids of one sample with the fragment marker inserted (L_0). labels: DEVICE int32
+ * [n_seq][num_heads + 1][seq_len]; row i of a sample is L_0 shifted left by i and filled up with
+ * pad_token, and in every column the labels beyond the column's last frag_token along the head
+ * axis are ignore_token (a column without a marker keeps only row 0; the paper leaves that
+ * case open). 0 <= num_heads <= 64, n_seq <= 65535; empty input is a no-op. Asynchronous on
+ * `cuda_stream`; returns SPEC_E_BADARG / SPEC_E_CUDA on bad arguments / a failed launch. */
+int spec_build_labels(const int32_t *tokens, int32_t n_seq, int32_t seq_len, int32_t num_heads,
+                      int32_t frag_token, int32_t pad_token, int32_t ignore_token, int32_t *labels,
+                      void *cuda_stream);
+
 /* The same operation as spec_op_linear for callers that cannot allocate device memory and so
  * have no scratch buffer to pass: code running where cudaMalloc is forbidden (inside a
  * real-time or safety-certified loop, under a framework whose memory pool is frozen or

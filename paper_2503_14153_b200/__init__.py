@@ -6,5 +6,5 @@ package does not load the shared library; the first call that needs it does, and
 loudly if it has not been built.
 """
 from .tree import build_tree, chain_tree  # noqa: F401
-from .binding import (SpecDecoder, SpecError, load_library, library_path, spec_op_linear, spec_op_linear_static,  # noqa: F401
+from .binding import (SpecDecoder, SpecError, load_library, library_path, spec_op_linear, spec_op_linear_static, spec_build_labels,  # noqa: F401
                       upload_weights, FLAG_KEEP_LOGITS, FLAG_SIMPLE_KERNELS)

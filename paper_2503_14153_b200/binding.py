@@ -26,7 +26,7 @@ TRACE_NAME_LEN = 32
 
 EXPORTS = ["spec_workspace_bytes", "spec_create", "spec_prefill", "spec_step", "spec_read_generated",
            "spec_destroy", "spec_last_error", "spec_query", "spec_debug_read", "spec_debug_read_kv",
-           "spec_op_linear", "spec_op_linear_scratch_floats", "spec_op_linear_static", "spec_set_option", "spec_trace_read", "spec_last_step_phase_ms", "spec_profile_kernel",
+           "spec_op_linear", "spec_op_linear_scratch_floats", "spec_op_linear_static", "spec_set_option", "spec_trace_read", "spec_build_labels", "spec_last_step_phase_ms", "spec_profile_kernel",
            "spec_profile_read"]
 
 
@@ -99,6 +99,9 @@ def load_library():
     lib.spec_set_option.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
     lib.spec_trace_read.restype = C.c_int
     lib.spec_trace_read.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+    lib.spec_build_labels.restype = C.c_int
+    lib.spec_build_labels.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                      C.c_void_p, C.c_void_p]
     lib.spec_op_linear_static.restype = C.c_int
     lib.spec_op_linear_static.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_void_p]
@@ -325,6 +328,19 @@ def spec_op_linear(x, w, ctas: int = 296):
     if rc != 0:
         raise SpecError(rc, "spec_op_linear failed")
     return y
+
+
+def spec_build_labels(tokens, num_heads: int, frag: int, pad: int, ignore: int):
+    """tokens: CUDA int32 tensor [n_seq, seq_len] -> labels [n_seq, num_heads + 1, seq_len] (Sec. III-C)."""
+    import torch
+    lib = load_library()
+    n_seq, seq_len = tokens.shape
+    labels = torch.empty((n_seq, num_heads + 1, seq_len), dtype=torch.int32, device=tokens.device)
+    rc = lib.spec_build_labels(tokens.data_ptr(), n_seq, seq_len, num_heads, frag, pad, ignore, labels.data_ptr(),
+                               torch.cuda.current_stream(tokens.device).cuda_stream)
+    if rc != 0:
+        raise SpecError(rc, "spec_build_labels failed")
+    return labels
 
 
 STATIC_SCRATCH_FLOATS = 2 << 20

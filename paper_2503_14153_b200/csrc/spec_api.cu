@@ -21,6 +21,7 @@
 #include "gemm_stream.cuh"
 #include "glue_tc.cuh"
 #include "kernels_simple.cuh"
+#include "labels.cuh"
 
 using namespace spec;
 
@@ -1148,6 +1149,17 @@ bool op_linear_args_ok(int32_t dtype, const void* x, const void* w, const float*
   return dtype == 1 && K % 64 == 0 && M % 16 == 0 && N >= 128 && ctas >= 1 && ctas <= 1024;
 }
 }  // namespace
+
+int spec_build_labels(const int32_t* tokens, int32_t n_seq, int32_t seq_len, int32_t num_heads, int32_t frag_token,
+                      int32_t pad_token, int32_t ignore_token, int32_t* labels, void* cuda_stream) {
+  if (n_seq == 0 || seq_len == 0) return SPEC_OK;
+  if (!tokens || !labels || n_seq < 0 || seq_len < 0 || num_heads < 0 || num_heads > LABEL_MAX_HEADS || n_seq > 65535)
+    return SPEC_E_BADARG;
+  dim3 grid((seq_len + LABEL_THREADS - 1) / LABEL_THREADS, n_seq);
+  build_labels_kernel<<<grid, LABEL_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(tokens, seq_len, num_heads, frag_token,
+                                                                                        pad_token, ignore_token, labels);
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_E_CUDA;
+}
 
 size_t spec_op_linear_scratch_floats(int32_t M, int32_t N, int32_t K, int32_t ctas) {
   GemmPlan g;

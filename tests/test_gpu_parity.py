@@ -159,3 +159,18 @@ def test_op_linear_fp32_vs_oracle_matmul(torch):
     y = spec_op_linear(torch.from_numpy(x).cuda(), torch.from_numpy(w).cuda()).cpu().numpy()
     ref = x.astype(np.float64) @ w.astype(np.float64).T
     assert np.abs(y - ref).max() / np.abs(ref).max() < 1e-5
+
+
+@pytest.mark.parametrize("n_seq,seq_len,K", [(1, 10, 3), (3, 8192, 10), (2, 257, 4), (1, 1, 10), (5, 1000, 0), (0, 16, 3)])
+def test_build_labels_vs_oracle(torch, n_seq, seq_len, K):
+    """Syntax-enriched labels (Sec. III-C): bit-exact against the oracle, ragged tails and empty input included."""
+    from oracle.labels import syntax_enriched_labels
+    from paper_2503_14153_b200 import spec_build_labels
+    frag, pad, ign = 32016, 32017, -100
+    rng = np.random.default_rng(seq_len * 31 + K)
+    toks = rng.integers(0, 32016, size=(n_seq, seq_len)).astype(np.int32)
+    toks[rng.random(toks.shape) < 0.15] = frag
+    got = spec_build_labels(torch.from_numpy(toks).cuda(), K, frag, pad, ign).cpu().numpy()
+    assert got.shape == (n_seq, K + 1, seq_len)
+    for i in range(n_seq):
+        assert np.array_equal(got[i], syntax_enriched_labels(toks[i], K, frag, pad, ign))
