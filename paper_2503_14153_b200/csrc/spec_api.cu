@@ -219,6 +219,12 @@ struct spec_ctx {
   bool prefilled = false;
   // timing: phase boundaries of the last step; optional per-launch timing of one kernel kind
   cudaEvent_t phase_ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  // enqueue-only steps: the committed lengths are copied to pinned host memory now and then, so
+  // the host's bounds on them stay tight without a synchronisation
+  int* h_n_pinned = nullptr;           // [max_batch], cudaHostAlloc
+  cudaEvent_t n_ev = nullptr;
+  bool n_copy_pending = false;
+  int n_copy_steps_after = 0;          // steps enqueued after the pending copy
   bool phase_valid = false;
   int profile_kind = 0;                 // SPEC_PROFILE_*
   std::vector<cudaEvent_t> prof_ev;     // pairs, reused every step
@@ -735,6 +741,7 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
   c->n_hi.assign(batch, 0);
   for (int b = 0; b < batch; ++b) c->n_hi[b] = offsets[b + 1] - offsets[b];
   c->n_lo = c->n_hi;
+  c->n_copy_pending = false;
   c->prefilled = true;
   return SPEC_OK;
 }
@@ -824,8 +831,28 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     r = check_status(c);   // synchronises
     if (r) return r;
     for (int b = 0; b < B; ++b) c->n_hi[b] = c->n_lo[b] = nn[b];
+    c->n_copy_pending = false;
   } else {
     for (int b = 0; b < B; ++b) { c->n_hi[b] += K + 1; c->n_lo[b] += 1; }
+    if (c->h_n_pinned && c->n_ev) {
+      if (c->n_copy_pending) {
+        c->n_copy_steps_after++;
+        if (cudaEventQuery(c->n_ev) == cudaSuccess) {
+          // the copy shows the lengths after an earlier step; every step since added 1..K+1 tokens
+          for (int b = 0; b < B; ++b) {
+            c->n_lo[b] = std::max(c->n_lo[b], c->h_n_pinned[b] + c->n_copy_steps_after);
+            c->n_hi[b] = std::min(c->n_hi[b], c->h_n_pinned[b] + c->n_copy_steps_after * (K + 1));
+          }
+          c->n_copy_pending = false;
+        }
+      }
+      if (!c->n_copy_pending &&
+          cudaMemcpyAsync(c->h_n_pinned, c->d_n, (size_t)B * sizeof(int), cudaMemcpyDeviceToHost, c->stream) == cudaSuccess &&
+          cudaEventRecord(c->n_ev, c->stream) == cudaSuccess) {
+        c->n_copy_pending = true;
+        c->n_copy_steps_after = 0;
+      }
+    }
   }
   return SPEC_OK;
 }
@@ -924,6 +951,9 @@ int spec_create(const spec_config* cfg, const spec_weights* w, const spec_tree* 
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_cand, 0, (size_t)cfg->max_batch * (c->K + 1) * c->kmax * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) { g_create_error = std::string("set-up copies: ") + cudaGetErrorString(e); delete c; return SPEC_E_CUDA; }
+  if (cudaHostAlloc(reinterpret_cast<void**>(&c->h_n_pinned), (size_t)cfg->max_batch * sizeof(int), cudaHostAllocDefault) != cudaSuccess) c->h_n_pinned = nullptr;
+  if (cudaEventCreateWithFlags(&c->n_ev, cudaEventDisableTiming) != cudaSuccess) c->n_ev = nullptr;
+  cudaGetLastError();
   *out = c;
   return SPEC_OK;
 }
@@ -970,6 +1000,8 @@ int spec_destroy(spec_ctx* c) {
   cudaStreamSynchronize(c->stream);
   for (int i = 0; i < 6; ++i) if (c->phase_ev[i]) cudaEventDestroy(c->phase_ev[i]);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+  if (c->n_ev) cudaEventDestroy(c->n_ev);
+  if (c->h_n_pinned) cudaFreeHost(c->h_n_pinned);
   delete c;
   return SPEC_OK;
 }
