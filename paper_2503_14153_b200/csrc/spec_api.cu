@@ -180,8 +180,9 @@ struct spec_ctx {
   int Mcap, cap, pages_per_seq, gen_cap, nsplit_attn, Nqkv, ntile_lm, topk_slice, topk_blocks;
   bool qkv_fused, keep_logits;
   bool pdl = true;                     // programmatic dependent launch between the kernels of a step
-  int gemm_ctas = SM_SLOTS;            // persistent CTAs of the weight-streaming GEMM
-  int l2_prefetch = 0;                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
+  int gemm_ctas = 288;                 // persistent CTAs of the weight-streaming GEMM (measured best; at most SM_SLOTS)
+  int l2_prefetch = 0;
+  int small_gemm_ctas = 192;           // CTAs of GEMMs with at most 48 weight tiles (Wo, down): fewer partial sums                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
   std::vector<int> h_parent, h_depth, h_rank;
   std::vector<int> n_hi, n_lo;         // host upper / lower bounds of the committed lengths
   std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, mw, mb;
@@ -415,7 +416,10 @@ const char* gemm_kind_name(int kind) {
 int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* const* mats, const int* rows, int kind,
              PartView* view) {
   GemmPlan g;
-  if (!plan_gemm(M, K, n_mats, rows, c->gemm_ctas, false, &g)) return c->fail(SPEC_E_BADARG, "unsupported linear shape");
+  int tiles_all = 0;
+  for (int i = 0; i < n_mats; ++i) tiles_all += (rows[i] + 127) / 128;
+  if (!plan_gemm(M, K, n_mats, rows, tiles_all <= 48 ? std::min(c->gemm_ctas, c->small_gemm_ctas) : c->gemm_ctas, false, &g))
+    return c->fail(SPEC_E_BADARG, "unsupported linear shape");
   if (plan_part_floats(g) > c->part_floats) return c->fail(SPEC_E_NOMEM, "partial-sum scratch too small");
   StreamTmaps tm{};
   for (int i = 0; i < n_mats; ++i) {
@@ -1036,6 +1040,9 @@ int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
     case SPEC_OPT_L2_PREFETCH:
       if (value < 0 || value > 64) return c->fail(SPEC_E_BADARG, "L2 prefetch depth out of range");
       c->l2_prefetch = value; return SPEC_OK;
+    case SPEC_OPT_SMALL_GEMM_CTAS:
+      if (value < 1 || value > SM_SLOTS) return c->fail(SPEC_E_BADARG, "out of range");
+      c->small_gemm_ctas = value; return SPEC_OK;
     case SPEC_OPT_TRACE:
       c->trace_on = value != 0;
       if (c->trace_on && c->trace_init.empty()) {
