@@ -221,7 +221,7 @@ medusa_act_tc(const PartView pv, int dpad, const bf16* __restrict__ hq_last, con
 }
 
 // Each row's kmax best (value desc, index asc) of this block's slice of the logits go to the
-// partial lists pk_val / pk_idx [block][rows][kmax]. grid (slices, rows); dynamic shared
+// partial lists pk_val / pk_idx [row][block][kmax]. grid (slices, rows); dynamic shared
 // memory: slice floats.
 __global__ void __launch_bounds__(256)
 topk_slices(const float* __restrict__ logits, int V, int rows_total, int slice, int kmax, float* __restrict__ pk_val,
@@ -245,7 +245,7 @@ topk_slices(const float* __restrict__ logits, int V, int rows_total, int slice, 
     __syncthreads();
     if (threadIdx.x == 0) {
       for (int w = 1; w < nw; ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
-      const size_t o = ((size_t)blockIdx.x * rows_total + row) * kmax + t;
+      const size_t o = ((size_t)row * gridDim.x + blockIdx.x) * kmax + t;
       pk_val[o] = bv;
       pk_idx[o] = bi;
       if (bi != 0x7fffffff) zs[bi - n0] = -INFINITY;

@@ -559,7 +559,7 @@ __global__ void medusa_resblock(const float* __restrict__ h_last, const T* const
 
 // z[row][n] = W_lm[n] . r[row] for MC rows (row = b*K + k) over this block's slice of the
 // vocabulary, kept in shared memory; then each row's kmax best (value desc, index asc) of
-// the slice go to the partial lists pk_val/pk_idx [block][rows][kmax].
+// the slice go to the partial lists pk_val/pk_idx [row][block][kmax].
 template <typename T, int MC>
 __global__ void medusa_lmhead_topk(const T* __restrict__ r, const T* __restrict__ Wlm, int rows_total, int V, int d,
                                    int slice, int kmax, float* __restrict__ pk_val, int* __restrict__ pk_idx,
@@ -605,7 +605,7 @@ __global__ void medusa_lmhead_topk(const T* __restrict__ r, const T* __restrict_
       for (int c = lane; c < n1 - n0; c += 32) if (better(z[c], n0 + c, bv, bi)) { bv = z[c]; bi = n0 + c; }
       warp_argmax(bv, bi);
       if (lane == 0) {
-        size_t o = ((size_t)blockIdx.x * rows_total + r0 + j) * kmax + t;
+        size_t o = ((size_t)(r0 + j) * gridDim.x + blockIdx.x) * kmax + t;
         pk_val[o] = bv;
         pk_idx[o] = bi;
         if (bi != 0x7fffffff) z[bi - n0] = -INFINITY;
@@ -634,8 +634,7 @@ __global__ void topk_merge(const float* __restrict__ pk_val, const int* __restri
   int* ix = reinterpret_cast<int*>(ms + total);
   int* head = ix + total;
   for (int c = threadIdx.x; c < total; c += blockDim.x) {
-    int blk = c / kmax, t = c % kmax;
-    size_t o = ((size_t)blk * rows_total + row) * kmax + t;
+    size_t o = (size_t)row * total + c;          // lists of a row are contiguous: [row][block][kmax]
     v[c] = pk_val[o];
     ix[c] = pk_idx[o];
   }

@@ -528,7 +528,7 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, cons
       int rws[3] = {HD, KD, KD};
       if ((r = run_gemm(c, u, M, d, 3, mats, rws, SPEC_PROFILE_QKV, &vq))) return r;
     }
-    KLAUNCH("rope_store_tc", rope_store_tc, dim3(M, M <= 128 ? 4 : 1), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope,
+    KLAUNCH("rope_store_tc", rope_store_tc, dim3(M, M <= 128 ? 8 : 1), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope,
             static_cast<bf16*>(c->d_q), static_cast<bf16*>(c->d_pool), c->geom, c->d_page_table, l, H);
     if ((r = launch_attention_tc(c, rows, R, l, n_hi_pass, n_lo_pass))) return r;
     PartView vo{};
