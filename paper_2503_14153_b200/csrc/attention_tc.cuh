@@ -37,7 +37,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-constexpr int ATTN_MAX_STAGES = 4;
+constexpr int ATTN_MAX_STAGES = 6;
 constexpr int ATTN_PT_CACHE = 256;
 constexpr int ATTN_MAX_SEQS = 16;
 
@@ -52,7 +52,8 @@ struct AttnTcArgs {
   int layer, H;
   int nsplit;           // KV splits (= gridDim.y), chosen by the host from its bound on the context length
   int tps;              // KV tiles per split
-  int stages;           // KV tiles in flight per CTA (2..ATTN_MAX_STAGES, a multiple of KG); sizes the shared memory
+  int stages;           // KV tiles in flight per CTA (2..ATTN_MAX_STAGES, at least KG); sizes the shared memory
+  int row_blocks;       // CTAs that share a (head, split): CTA j of them owns query rows [16 NW j, 16 NW (j+1)); > 1 only with nsplit == 1
   int n_lo[ATTN_MAX_SEQS];   // host's lower bound of each sequence's committed length: keys below it
                              // were written by earlier steps and may be fetched before the dependency wait
   float scale_log2;     // log2(e) / sqrt(head_dim)
@@ -100,7 +101,8 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rg = warp % NW, kg = warp / NW;
-  const int h = blockIdx.x, sp = blockIdx.y, b = blockIdx.z;
+  const int h = blockIdx.x, sp = blockIdx.y / a.row_blocks, b = blockIdx.z;
+  const int row0 = (blockIdx.y % a.row_blocks) * NW * 16;        // first query row of this CTA
   const int H = a.H, kvh = h / (H / a.g.n_kv_heads);
   const int nsplit = a.nsplit, tps = a.tps;
   const int t0 = sp * tps;
@@ -138,7 +140,7 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   if (threadIdx.x == 0) trace_mark_min(tr, 2);
   // sequence state, ancestor sets and the Q tile are independent loads: one trip for all of them
   const int R = a.rows.R, cnt = a.rows.cnt[b], n = a.rows.n[b];
-  const int i0 = rg * 16 + (lane >> 2), i1 = i0 + 8;        // this thread's two query rows
+  const int i0 = row0 + rg * 16 + (lane >> 2), i1 = i0 + 8;  // this thread's two query rows
   uint32_t anc0[4], anc1[4];
 #pragma unroll
   for (int w = 0; w < 4; ++w) { anc0[w] = a.rows.anc[i0 * 4 + w]; anc1[w] = a.rows.anc[i1 * 4 + w]; }
@@ -150,7 +152,7 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
     const int c = threadIdx.x + k * NTHR;
     const int r = c / (HD / 8), ch = c % (HD / 8);
     qv[k] = make_uint4(0, 0, 0, 0);
-    if (c < QC && r < R) qv[k] = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + r) * H * HD + h * HD + ch * 8);
+    if (c < QC && row0 + r < R) qv[k] = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + row0 + r) * H * HD + h * HD + ch * 8);
   }
   const int S = n + cnt;
   const int M = a.rows.B * R;
@@ -172,7 +174,7 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   for (int k = 0; k < PER; ++k) {
     const int c = threadIdx.x + k * NTHR;
     const int r = c / (HD / 8), ch = c % (HD / 8);
-    if (c < QC) *reinterpret_cast<uint4*>(qs + r * ROWB + ((ch ^ (r & 7)) << 4)) = (r < cnt) ? qv[k] : make_uint4(0, 0, 0, 0);
+    if (c < QC) *reinterpret_cast<uint4*>(qs + r * ROWB + ((ch ^ (r & 7)) << 4)) = (row0 + r < cnt) ? qv[k] : make_uint4(0, 0, 0, 0);
   }
   __syncthreads();
 
@@ -310,36 +312,43 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
     lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
     lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
   }
-  if (KG == 2) {
-    // merge the two key groups' states through the (now idle) KV buffers
+  if (KG > 1) {
+    // merge the key groups' states through the (now idle) KV buffers: groups 1.. leave theirs,
+    // group 0 adds them in group order
     float* ex = reinterpret_cast<float*>(ks);
     constexpr int GT = NW * 32;                                // threads per key group
+    constexpr int SLOT = (HD / 2 + 4) * GT;                    // floats per group state
     const int gt = rg * 32 + lane;
-    if (kg == 1) {
+    if (kg > 0) {
+      float* my = ex + (size_t)(kg - 1) * SLOT;
 #pragma unroll
       for (int d = 0; d < HD / 8; ++d)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) ex[(d * 4 + e) * GT + gt] = o[d][e];
-      ex[(HD / 2 + 0) * GT + gt] = mrow[0]; ex[(HD / 2 + 1) * GT + gt] = mrow[1];
-      ex[(HD / 2 + 2) * GT + gt] = lrow[0]; ex[(HD / 2 + 3) * GT + gt] = lrow[1];
+        for (int e = 0; e < 4; ++e) my[(d * 4 + e) * GT + gt] = o[d][e];
+      my[(HD / 2 + 0) * GT + gt] = mrow[0]; my[(HD / 2 + 1) * GT + gt] = mrow[1];
+      my[(HD / 2 + 2) * GT + gt] = lrow[0]; my[(HD / 2 + 3) * GT + gt] = lrow[1];
     }
     __syncthreads();
     if (kg == 0) {
-      float w0[2], w1[2];
+#pragma unroll 1
+      for (int g2 = 1; g2 < KG; ++g2) {
+        const float* th = ex + (size_t)(g2 - 1) * SLOT;
+        float w0[2], w1[2];
 #pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const float m1 = ex[(HD / 2 + r) * GT + gt], l1 = ex[(HD / 2 + 2 + r) * GT + gt];
-        const float mm = fmaxf(mrow[r], m1);
-        const float base = (mm == -INFINITY) ? 0.f : mm;
-        w0[r] = exp2f(mrow[r] - base);
-        w1[r] = exp2f(m1 - base);
-        mrow[r] = mm;
-        lrow[r] = lrow[r] * w0[r] + l1 * w1[r];
+        for (int r = 0; r < 2; ++r) {
+          const float m1 = th[(HD / 2 + r) * GT + gt], l1 = th[(HD / 2 + 2 + r) * GT + gt];
+          const float mm = fmaxf(mrow[r], m1);
+          const float base = (mm == -INFINITY) ? 0.f : mm;
+          w0[r] = exp2f(mrow[r] - base);
+          w1[r] = exp2f(m1 - base);
+          mrow[r] = mm;
+          lrow[r] = lrow[r] * w0[r] + l1 * w1[r];
+        }
+#pragma unroll
+        for (int d = 0; d < HD / 8; ++d)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) o[d][e] = o[d][e] * w0[e >> 1] + th[(d * 4 + e) * GT + gt] * w1[e >> 1];
       }
-#pragma unroll
-      for (int d = 0; d < HD / 8; ++d)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) o[d][e] = o[d][e] * w0[e >> 1] + ex[(d * 4 + e) * GT + gt] * w1[e >> 1];
     }
   }
   if (nsplit == 1) {

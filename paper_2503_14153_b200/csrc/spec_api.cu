@@ -481,10 +481,15 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
   // into at most one split per resident CTA slot, eight tiles or more each
   const int slots1 = std::max(1, std::min(c->nsplit_attn, (SM_SLOTS / 2) / (H * c->B)));
   a.nsplit = tiles_hi <= 12 ? 1 : std::min(slots1, (tiles_hi + 7) / 8);
-  a.stages = ATTN_MAX_STAGES;
+  a.stages = 4;
   a.tps = (tiles_hi + a.nsplit - 1) / a.nsplit;
-  dim3 grid(H, a.nsplit, c->B);
+  a.row_blocks = 1;
   int nw = (R + 15) / 16;
+  // short context and few sequences: a CTA per 16 query rows, its six warps taking a KV tile each,
+  // so that a head's work spreads over several SMs instead of one
+  const bool row_mode = a.nsplit == 1 && nw > 1 && nw <= 4 && H * c->B * nw <= SM_SLOTS / 2;
+  if (row_mode) { a.row_blocks = nw; a.stages = 6; }
+  dim3 grid(H, a.nsplit * a.row_blocks, c->B);
 #define ATTN_CASE(HDV, NWV, KGV)                                                                         \
   {                                                                                                    \
     size_t sm = attention_tc_smem(HDV, NWV, a.stages);                                                 \
@@ -496,9 +501,11 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
     // up to 64 rows: two key groups of warps per CTA; more rows: one
     ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
     if (D == 128) {
-      if (nw <= 1) ATTN_CASE(128, 1, 2) else if (nw <= 2) ATTN_CASE(128, 2, 2) else if (nw <= 4) ATTN_CASE(128, 4, 2) else ATTN_CASE(128, 8, 1)
+      if (row_mode) ATTN_CASE(128, 1, 6)
+      else if (nw <= 1) ATTN_CASE(128, 1, 2) else if (nw <= 2) ATTN_CASE(128, 2, 2) else if (nw <= 4) ATTN_CASE(128, 4, 2) else ATTN_CASE(128, 8, 1)
     } else {
-      if (nw <= 1) ATTN_CASE(64, 1, 2) else if (nw <= 2) ATTN_CASE(64, 2, 2) else if (nw <= 4) ATTN_CASE(64, 4, 2) else ATTN_CASE(64, 8, 1)
+      if (row_mode) ATTN_CASE(64, 1, 6)
+      else if (nw <= 1) ATTN_CASE(64, 1, 2) else if (nw <= 2) ATTN_CASE(64, 2, 2) else if (nw <= 4) ATTN_CASE(64, 4, 2) else ATTN_CASE(64, 8, 1)
     }
   }
 #undef ATTN_CASE
