@@ -79,6 +79,19 @@ class ClockSampler:
         return out
 
 
+def aggregate_replicas(seconds: float, units: float, world: int, device="cpu"):
+    """Whole-job figures of `world` independent replicas: the slowest rank's time (max) and all ranks'
+    units (sum). With world > 1 the default process group must be initialised."""
+    import torch
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    u = torch.tensor([float(units)], dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
 def algorithmic_bytes(cfg, n_ctx: int, T: int):
     """Bytes one step must read: verify = layer weights + lm_head + cached K/V + tree activations;
     the whole step adds the head matrices and the heads' pass over lm_head."""
@@ -252,12 +265,7 @@ def main():
     tokens = len(gen) - n_before
     n_ctx_mid = cfg.prompt_len + n_before + tokens // 2
     phase = dec.phase_ms()
-    t_ms = torch.tensor([ms], dtype=torch.float64, device=dev)
-    t_tok = torch.tensor([float(tokens)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-        dist.all_reduce(t_tok, op=dist.ReduceOp.SUM)
-    ms_max, tokens_all = float(t_ms.item()), float(t_tok.item())
+    ms_max, tokens_all = aggregate_replicas(ms, tokens, world, dev)
     value = tokens_all / (ms_max * 1e-3)
     ms_per_step = ms_max / args.steps
 
@@ -296,14 +304,10 @@ def main():
             e_tokens += int(cnt[0])
         torch.cuda.synchronize()
         e_s = time.perf_counter() - t0
-        t_e = torch.tensor([e_s], dtype=torch.float64, device=dev)
-        t_et = torch.tensor([float(e_tokens)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t_e, op=dist.ReduceOp.MAX)
-            dist.all_reduce(t_et, op=dist.ReduceOp.SUM)
-        out["e2e"] = {"value": float(t_et.item()) / float(t_e.item()), "unit": UNIT,
+        e_max, e_tok_all = aggregate_replicas(e_s, e_tokens, world, dev)
+        out["e2e"] = {"value": e_tok_all / e_max, "unit": UNIT,
                       "h2d_bytes_per_step": int(keep.nbytes), "d2h_bytes_per_step": int((K + 1) * 4 + 4 + 4 + 16),
-                      "ms_per_step": float(t_e.item()) * 1e3 / args.steps}
+                      "ms_per_step": e_max * 1e3 / args.steps}
 
         # ---------------- dominant kernel: gate/up projection with fused SwiGLU ----------------
         dec.profile_kernel(B.PROFILE_GATE_UP)
