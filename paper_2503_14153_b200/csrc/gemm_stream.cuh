@@ -76,8 +76,9 @@ template <int MT, int DEEP> struct StreamCfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-__device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
+__device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int x, int y, uint64_t policy) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile.L2::cache_hint [%0, {%1, %2}], %3;"
+               ::"l"(tmap), "r"(x), "r"(y), "l"(policy) : "memory");
 }
 
 struct GsUnit {
@@ -160,7 +161,7 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
         if (n_pf > p.l2_prefetch) n_pf = p.l2_prefetch;
         for (int i = 0; i < n_pf; ++i) {
           GsUnit w = gs_decode(p, lo + n_pre + i);
-          tma_prefetch_l2_2d(&tm.a[w.mat], w.kc * Cfg::BK, w.row0);
+          tma_prefetch_l2_2d(&tm.a[w.mat], w.kc * Cfg::BK, w.row0, wpol);
         }
       }
       pdl_wait();
