@@ -36,7 +36,7 @@ class ModelConfig:
 
     @property
     def kmax(self) -> int:
-        return max(self.topk)
+        return max(self.topk) if self.topk else 1
 
 
 _TINY = ModelConfig(

@@ -174,3 +174,39 @@ def test_build_labels_vs_oracle(torch, n_seq, seq_len, K):
     assert got.shape == (n_seq, K + 1, seq_len)
     for i in range(n_seq):
         assert np.array_equal(got[i], syntax_enriched_labels(toks[i], K, frag, pad, ign))
+
+
+def test_error_returns_and_degenerate_shapes(torch):
+    """Calls out of order and sequences that run out of room return error codes (nothing faults); a
+    one-token prompt and a model without extra heads (every step emits exactly the root) still decode."""
+    from paper_2503_14153_b200 import SpecDecoder, SpecError, build_tree, chain_tree, upload_weights
+    from tests_lockstep import run_lockstep
+    cfg = get_config("c0")
+    w = draw_weights(cfg)
+    dw = upload_weights(cfg, w)
+    tree = build_tree(cfg.topk, cfg.tree_nodes)
+    dec = SpecDecoder(cfg, dw, tree, max_seq=40)
+    with pytest.raises(SpecError) as e:
+        dec.step()
+    assert e.value.code == -7                      # step before prefill
+    with pytest.raises(SpecError) as e:
+        dec.prefill(draw_prompt(cfg, 39))          # leaves no room to generate within max_seq
+    assert e.value.code == -4
+    dec.prefill(draw_prompt(cfg, 30))
+    with pytest.raises(SpecError) as e:
+        for _ in range(20):
+            dec.step()
+    assert e.value.code == -4                      # ran into max_seq after a few steps
+    dec.close()
+    # one-token prompt
+    rep = run_lockstep(cfg, w, tree, draw_prompt(cfg, 1), 8, TOL_FP32)
+    assert rep.steps > 0
+    # no extra heads: the tree is the root alone
+    cfg0 = get_config("c0", n_medusa=0, topk=(), tree_nodes=1)
+    w0 = draw_weights(cfg0)
+    dec = SpecDecoder(cfg0, upload_weights(cfg0, w0), chain_tree(1), max_seq=64)
+    dec.prefill(draw_prompt(cfg0, 9))
+    for _ in range(3):
+        tok, cnt = dec.step()
+        assert int(cnt[0]) == 1
+    dec.close()
