@@ -46,16 +46,10 @@ struct StreamGemmParams {
   int mat_col0[GS_MAX_MATS];        // first logical output column of each matrix
   int n_tiles;
   SegMap seg;
-  int tile_granular;                // 1: runs are cut at tile boundaries (argmax / logits epilogue)
   int l2_prefetch;                  // units to request into L2 beyond the ring before the dependency wait
   // partial sums: part[slot][m][n_tiles*128] (padded column space: tile nt owns columns [128 nt, 128 nt + 128))
   float* part;
   size_t slot_stride;
-  // tile-granular epilogue: per-(row, tile, lane quarter) argmax partials and optional logits [M][N]
-  float* logits;
-  int ld_logits;
-  float* pval;
-  int* pidx;
   int* status;
   unsigned long long* trace;        // optional timeline slot (see KTrace); [2] first operands landed, [3] last MMA issued
 };
@@ -118,15 +112,7 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x;
   const int KC = p.seg.KC;
-  int lo, hi;
-  if (p.tile_granular) {
-    const int nt_all = p.n_tiles * p.seg.m_tiles;
-    lo = (int)(((long long)c * nt_all) / gridDim.x) * KC;
-    hi = (int)(((long long)(c + 1) * nt_all) / gridDim.x) * KC;
-  } else {
-    lo = p.seg.lo(c);
-    hi = p.seg.lo(c + 1);
-  }
+  const int lo = p.seg.lo(c), hi = p.seg.lo(c + 1);
 
   pdl_launch_dependents();
 
@@ -236,57 +222,30 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * MT);
       const int m0 = mt * MT;
-      if (!p.tile_granular) {
-        const int slot = c - p.seg.owner(t * KC);
-        float* dst = p.part + (size_t)slot * p.slot_stride + (size_t)nt * 128 + q * 32 + lane;
-        const size_t ld = (size_t)p.n_tiles * 128;
-        if (MT >= 32) {
-          // all loads of the accumulator are issued before the first store
-          uint32_t r[MT >= 32 ? MT / 32 : 1][32];
+      const int slot = c - p.seg.owner(t * KC);
+      float* dst = p.part + (size_t)slot * p.slot_stride + (size_t)nt * 128 + q * 32 + lane;
+      const size_t ld = (size_t)p.n_tiles * 128;
+      if (MT >= 32) {
+        // all loads of the accumulator are issued before the first store
+        uint32_t r[MT >= 32 ? MT / 32 : 1][32];
 #pragma unroll
-          for (int g = 0; g < MT / 32; ++g) tmem_ld32(taddr + g * 32, r[g]);
-          tmem_ld_wait();
+        for (int g = 0; g < MT / 32; ++g) tmem_ld32(taddr + g * 32, r[g]);
+        tmem_ld_wait();
 #pragma unroll
-          for (int g = 0; g < MT / 32; ++g)
+        for (int g = 0; g < MT / 32; ++g)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int m = m0 + g * 32 + j;
-              if (m < p.M) dst[(size_t)m * ld] = __uint_as_float(r[g][j]);
-            }
-        } else {
-          uint32_t r[16];
-          tmem_ld16(taddr, r);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int m = m0 + j;
-            if (m < p.M) dst[(size_t)m * ld] = __uint_as_float(r[j]);
+          for (int j = 0; j < 32; ++j) {
+            const int m = m0 + g * 32 + j;
+            if (m < p.M) dst[(size_t)m * ld] = __uint_as_float(r[g][j]);
           }
-        }
       } else {
-        int mat = 0;
-        for (int i = 1; i < p.n_mats; ++i) if (nt >= p.mat_tile0[i]) mat = i;
-        const int row = (nt - p.mat_tile0[mat]) * 128 + q * 32 + lane;
-        const bool valid = row < p.mat_rows[mat];
-        const int n = p.mat_col0[mat] + row;
-#pragma unroll 1
-        for (int col = 0; col < MT; col += 16) {
-          uint32_t r[16];
-          tmem_ld16(taddr + col, r);
-          tmem_ld_wait();
+        uint32_t r[16];
+        tmem_ld16(taddr, r);
+        tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int m = m0 + col + j;
-            float v = valid ? __uint_as_float(r[j]) : -INFINITY;
-            if (p.logits && valid && m < p.M) p.logits[(size_t)m * p.ld_logits + n] = v;
-            int idx = valid ? n : 0x7fffffff;
-            warp_argmax(v, idx);
-            if (lane == 0 && m < p.M) {
-              const size_t o = ((size_t)m * p.n_tiles + nt) * 4 + q;
-              p.pval[o] = v;
-              p.pidx[o] = idx;
-            }
-          }
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + j;
+          if (m < p.M) dst[(size_t)m * ld] = __uint_as_float(r[j]);
         }
       }
       tc_fence_before();

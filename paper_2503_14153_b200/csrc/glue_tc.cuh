@@ -254,6 +254,80 @@ topk_slices(const float* __restrict__ logits, int V, int rows_total, int slice, 
   }
 }
 
+// lm_head consumers of the GEMM's partial sums. argmax_partials_tc: row m, vocabulary slice
+// blockIdx.y of gridDim.y: logits = sum of the slots (written out when `logits` is given), the
+// slice's best (value desc, index asc) goes to pval / pidx [m][gridDim.y].
+__global__ void __launch_bounds__(256)
+argmax_partials_tc(const PartView pv, int V, float* __restrict__ logits, float* __restrict__ pval, int* __restrict__ pidx,
+                   unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  const int m = blockIdx.x, nsl = gridDim.y;
+  const int v4 = (V + 3) >> 2;
+  const int per = (v4 + nsl - 1) / nsl;
+  const int c_lo = blockIdx.y * per, c_hi = min(v4, c_lo + per);
+  float bv = -INFINITY; int bi = 0x7fffffff;
+  for (int c4 = c_lo + threadIdx.x; c4 < c_hi; c4 += blockDim.x) {
+    const float4 a = part_sum4(pv, m, c4 * 4);
+    const float z[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = c4 * 4 + j;
+      if (n < V) {
+        if (logits) logits[(size_t)m * V + n] = z[j];
+        if (better(z[j], n, bv, bi)) { bv = z[j]; bi = n; }
+      }
+    }
+  }
+  __shared__ float sv[8];
+  __shared__ int si[8];
+  warp_argmax(bv, bi);
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
+    pval[(size_t)m * nsl + blockIdx.y] = bv;
+    pidx[(size_t)m * nsl + blockIdx.y] = bi;
+  }
+}
+
+// topk_slices over the partial sums of the heads' lm_head GEMM instead of materialised logits.
+__global__ void __launch_bounds__(256)
+topk_slices_tc(const PartView pv, int V, int rows_total, int slice, int kmax, float* __restrict__ pk_val,
+               int* __restrict__ pk_idx, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  extern __shared__ float zs[];
+  const int row = blockIdx.y, n0 = blockIdx.x * slice, n1 = min(n0 + slice, V);    // slice % 4 == 0
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  for (int c4 = threadIdx.x; c4 * 4 < n1 - n0; c4 += blockDim.x) {
+    const float4 a = part_sum4(pv, row, n0 + c4 * 4);
+    zs[c4 * 4] = a.x; zs[c4 * 4 + 1] = a.y; zs[c4 * 4 + 2] = a.z; zs[c4 * 4 + 3] = a.w;
+  }
+  __syncthreads();
+  __shared__ float sv[8];
+  __shared__ int si[8];
+  for (int t = 0; t < kmax; ++t) {
+    float bv = -INFINITY; int bi = 0x7fffffff;
+    for (int c = threadIdx.x; c < n1 - n0; c += blockDim.x) if (better(zs[c], n0 + c, bv, bi)) { bv = zs[c]; bi = n0 + c; }
+    warp_argmax(bv, bi);
+    if (lane == 0) { sv[warp] = bv; si[warp] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 1; w < nw; ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
+      const size_t o = ((size_t)row * gridDim.x + blockIdx.x) * kmax + t;
+      pk_val[o] = bv;
+      pk_idx[o] = bi;
+      if (bi != 0x7fffffff) zs[bi - n0] = -INFINITY;
+    }
+    __syncthreads();
+  }
+}
+
 // Finishes the per-row argmax from the per-(tile, lane quarter) partials of the lm_head
 // epilogue: one CTA per row, result in pval2[m] / pidx2[m].
 __global__ void __launch_bounds__(256)

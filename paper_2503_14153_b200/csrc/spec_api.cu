@@ -104,7 +104,7 @@ struct GemmPlan {
   int MT, grid;
 };
 
-bool plan_gemm(int M, int K, int n_mats, const int* rows, int g_max, bool tile_granular, GemmPlan* out) {
+bool plan_gemm(int M, int K, int n_mats, const int* rows, int g_max, GemmPlan* out) {
   if (M < 1 || K < 64 || K % 64 || n_mats < 1 || n_mats > GS_MAX_MATS || g_max < 1) return false;
   GemmPlan& g = *out;
   g = GemmPlan{};
@@ -125,9 +125,7 @@ bool plan_gemm(int M, int K, int n_mats, const int* rows, int g_max, bool tile_g
   long long total = (long long)tiles * p.seg.m_tiles * p.seg.KC;
   if (total > 0x3fffffff || (total + 1) * (long long)g_max >= 0x7fffffffLL) return false;
   p.seg.total = (int)total;
-  p.tile_granular = tile_granular ? 1 : 0;
-  long long cap = tile_granular ? (long long)tiles * p.seg.m_tiles : total;
-  g.grid = (int)std::min<long long>(g_max, cap);
+  g.grid = (int)std::min<long long>(g_max, total);
   p.seg.G = g.grid;
   return true;
 }
@@ -208,7 +206,6 @@ struct spec_ctx {
   unsigned int* d_attn_arrive = nullptr;
   float* d_pval2 = nullptr;            // finished per-row argmax (tensor-core path)
   int* d_pidx2 = nullptr;
-  float* d_head_logits = nullptr;      // [B*K][vocab] logits of the extra heads (tensor-core path)
   int trace_n = 0;
   std::vector<std::string> trace_names;
   std::vector<unsigned long long> trace_init;
@@ -296,8 +293,8 @@ size_t carve(spec_ctx* c, void* base) {
   if (64 % f.page_size == 0) c->cap = (int)round_up(c->cap, 64);   // whole 64-key attention tiles
   c->pages_per_seq = c->cap / f.page_size;
   c->gen_cap = f.max_seq + K + 1;
-  c->ntile_lm = c->tc ? ((V + 127) / 128) * 4 : 1;   // argmax partials per row (tile x lane quarter)
-  c->topk_slice = (V + SM_SLOTS - 1) / SM_SLOTS;
+  c->ntile_lm = c->tc ? 8 : 1;   // argmax partials per row (vocabulary slices)
+  c->topk_slice = ((V + SM_SLOTS - 1) / SM_SLOTS + 3) / 4 * 4;
   c->topk_blocks = (V + c->topk_slice - 1) / c->topk_slice;
   c->nsplit_attn = c->tc ? std::max(1, std::min(16, (SM_SLOTS / 2) / (f.n_heads * B))) : 1;   // most KV splits a launch may use
   int Mlog = (int)round_up((size_t)B * T, 16);
@@ -308,7 +305,6 @@ size_t carve(spec_ctx* c, void* base) {
   c->d_trace = b.take<unsigned long long>((size_t)TRACE_CAP * 4);
   c->d_attn_arrive = b.take<unsigned int>((size_t)B * f.n_heads);
   c->d_pval2 = b.take<float>(c->Mcap); c->d_pidx2 = b.take<int>(c->Mcap);
-  c->d_head_logits = c->tc ? b.take<float>(round_up((size_t)B * (K ? K : 1), 16) * V, 1024) : nullptr;
   c->d_n = b.take<int>(B); c->d_cnt = b.take<int>(B); c->d_n_old = b.take<int>(B); c->d_root = b.take<int>(B);
   c->d_count = b.take<int>(B); c->d_path = b.take<int>((size_t)B * (K + 1)); c->d_out_tok = b.take<int>((size_t)B * (K + 1));
   c->d_gen_cnt = b.take<int>(B); c->d_gen_log = b.take<int>((size_t)B * c->gen_cap);
@@ -331,10 +327,14 @@ size_t carve(spec_ctx* c, void* base) {
         int KD = f.n_kv_heads * f.head_dim;
         int r_qkv[3] = {HD, KD, KD}, r_o[1] = {d}, r_gu[2] = {F, F}, r_dn[1] = {d};
         GemmPlan g;
-        if (plan_gemm((int)m, d, 3, r_qkv, SM_SLOTS, false, &g)) pf = std::max(pf, plan_part_floats(g));
-        if (plan_gemm((int)m, HD, 1, r_o, SM_SLOTS, false, &g)) pf = std::max(pf, plan_part_floats(g));
-        if (plan_gemm((int)m, d, 2, r_gu, SM_SLOTS, false, &g)) pf = std::max(pf, plan_part_floats(g));
-        if (plan_gemm((int)m, F, 1, r_dn, SM_SLOTS, false, &g)) pf = std::max(pf, plan_part_floats(g));
+        if (plan_gemm((int)m, d, 3, r_qkv, SM_SLOTS, &g)) pf = std::max(pf, plan_part_floats(g));
+        if (plan_gemm((int)m, HD, 1, r_o, SM_SLOTS, &g)) pf = std::max(pf, plan_part_floats(g));
+        if (plan_gemm((int)m, d, 2, r_gu, SM_SLOTS, &g)) pf = std::max(pf, plan_part_floats(g));
+        if (plan_gemm((int)m, F, 1, r_dn, SM_SLOTS, &g)) pf = std::max(pf, plan_part_floats(g));
+        int r_lm[1] = {V};
+        if (plan_gemm((int)m, d, 1, r_lm, SM_SLOTS, &g)) pf = std::max(pf, plan_part_floats(g));
+        int r_hd[GS_MAX_MATS] = {d, d, d, d};
+        if (plan_gemm((int)m, d, GS_MAX_MATS, r_hd, SM_SLOTS, &g)) pf = std::max(pf, plan_part_floats(g));
       } else {
         pf = std::max(pf, std::max(m * (size_t)c->Nqkv, 2 * m * (size_t)F));
       }
@@ -418,7 +418,7 @@ int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* c
   GemmPlan g;
   int tiles_all = 0;
   for (int i = 0; i < n_mats; ++i) tiles_all += (rows[i] + 127) / 128;
-  if (!plan_gemm(M, K, n_mats, rows, tiles_all <= 48 ? std::min(c->gemm_ctas, c->small_gemm_ctas) : c->gemm_ctas, false, &g))
+  if (!plan_gemm(M, K, n_mats, rows, tiles_all <= 48 ? std::min(c->gemm_ctas, c->small_gemm_ctas) : c->gemm_ctas, &g))
     return c->fail(SPEC_E_BADARG, "unsupported linear shape");
   if (plan_part_floats(g) > c->part_floats) return c->fail(SPEC_E_NOMEM, "partial-sum scratch too small");
   StreamTmaps tm{};
@@ -616,29 +616,6 @@ int forward_layers(spec_ctx* c, int R, bool chain, const int* n_hi_pass, const i
   return SPEC_OK;
 }
 
-// lm_head on the tensor cores over `M` bf16 operand rows at `src`: each CTA owns whole weight
-// tiles, leaves per-(row, tile, lane quarter) argmax partials and, if asked, the logits.
-int lm_head_gemm_tc(spec_ctx* c, const void* src, int M, float* logits) {
-  const spec_config& f = c->cfg;
-  GemmPlan g;
-  int rws[1] = {f.vocab};
-  if (!plan_gemm(M, f.d_model, 1, rws, c->gemm_ctas, true, &g)) return c->fail(SPEC_E_BADARG, "unsupported lm_head shape");
-  StreamTmaps tm{};
-  const CUtensorMap* ta = c->tmap(c->lm_head, f.vocab, f.d_model, 128);
-  const CUtensorMap* tb = c->tmap(src, std::max<size_t>(round_up(M, 16), g.MT), f.d_model, g.MT);
-  if (!ta || !tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed");
-  tm.a[0] = *ta; tm.b = *tb;
-  g.p.logits = logits; g.p.ld_logits = f.vocab;
-  g.p.pval = c->d_pval; g.p.pidx = c->d_pidx;
-  g.p.l2_prefetch = c->l2_prefetch;
-  g.p.status = c->d_status;
-  g.p.trace = c->next_trace("gemm_lm_head");
-  cudaError_t e = launch_gs(c->stream, c->pdl, g, tm);
-  c->launches++;
-  if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_stream lm_head launch: ") + cudaGetErrorString(e));
-  return SPEC_OK;
-}
-
 // Extra decoding heads on the tensor cores: residual blocks (head matrices stacked along the
 // output dimension, up to four per launch), shared lm_head, per-head top-k.
 int heads_tc(spec_ctx* c, const int* ov) {
@@ -656,10 +633,15 @@ int heads_tc(spec_ctx* c, const int* ov) {
     KLAUNCH("medusa_act_tc", medusa_act_tc, dim3(B * nk, 4), dim3(256), 0, pv, dpad, (const bf16*)c->d_hq_last,
             reinterpret_cast<const bf16* const*>(c->d_mb), static_cast<bf16*>(c->d_r), K, k0, nk, d);
   }
-  int r = lm_head_gemm_tc(c, c->d_r, rows_total, c->d_head_logits);
-  if (r) return r;
-  KLAUNCH("topk_slices", topk_slices, dim3(c->topk_blocks, rows_total), dim3(256), (size_t)c->topk_slice * sizeof(float),
-          (const float*)c->d_head_logits, f.vocab, rows_total, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
+  PartView pl{};
+  {
+    const void* mats[1] = {c->lm_head};
+    int rws[1] = {f.vocab};
+    int r = run_gemm(c, c->d_r, rows_total, d, 1, mats, rws, SPEC_PROFILE_OFF, &pl);
+    if (r) return r;
+  }
+  KLAUNCH("topk_slices_tc", topk_slices_tc, dim3(c->topk_blocks, rows_total), dim3(256), (size_t)c->topk_slice * sizeof(float),
+          pl, f.vocab, rows_total, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
   size_t sm2 = (size_t)c->topk_blocks * kmax * 8 + (size_t)c->topk_blocks * 4;
   KLAUNCH("topk_merge", topk_merge, dim3(rows_total), dim3(256), sm2, (const float*)c->d_pk_val, (const int*)c->d_pk_idx,
           c->topk_blocks, rows_total, K, kmax, (const int*)c->d_root, ov, c->d_cand);
@@ -671,9 +653,15 @@ template <typename T>
 int lm_head_argmax(spec_ctx* c, const T* src, int M) {
   const spec_config& f = c->cfg;
   if (c->tc) {
-    int r = lm_head_gemm_tc(c, src, M, c->keep_logits ? c->d_logits : nullptr);
+    PartView pl{};
+    const void* mats[1] = {c->lm_head};
+    int rws[1] = {f.vocab};
+    int r = run_gemm(c, src, M, f.d_model, 1, mats, rws, SPEC_PROFILE_OFF, &pl);
     if (r) return r;
-    KLAUNCH("argmax_finish", argmax_finish, dim3(M), dim3(256), 0, (const float*)c->d_pval, (const int*)c->d_pidx, c->ntile_lm,
+    const int NSL = c->ntile_lm;
+    KLAUNCH("argmax_partials_tc", argmax_partials_tc, dim3(M, NSL), dim3(256), 0, pl, f.vocab,
+            c->keep_logits ? c->d_logits : (float*)nullptr, c->d_pval, c->d_pidx);
+    KLAUNCH("argmax_finish", argmax_finish, dim3(M), dim3(256), 0, (const float*)c->d_pval, (const int*)c->d_pidx, NSL,
             c->d_pval2, c->d_pidx2);
   } else {
     int r = linear_simple<T>(c, src, f.d_model, static_cast<const T*>(c->lm_head), c->d_logits, f.vocab, M, f.vocab, f.d_model);
@@ -1171,7 +1159,7 @@ int op_linear_bf16(const void* x, const void* w, float* y, int M, int N, int K, 
                    size_t scratch_floats, cudaStream_t st) {
   GemmPlan g;
   int rws[1] = {N};
-  if (!plan_gemm(M, K, 1, rws, ctas, false, &g)) return SPEC_E_BADARG;
+  if (!plan_gemm(M, K, 1, rws, ctas, &g)) return SPEC_E_BADARG;
   StreamTmaps tm{};
   if (!make_tmap(&tm.a[0], w, N, K, 128) || !make_tmap(&tm.b, x, M, K, g.MT)) return SPEC_E_CUDA;
   g.p.part = scratch;
@@ -1210,7 +1198,7 @@ int spec_build_labels(const int32_t* tokens, int32_t n_seq, int32_t seq_len, int
 size_t spec_op_linear_scratch_floats(int32_t M, int32_t N, int32_t K, int32_t ctas) {
   GemmPlan g;
   int rws[1] = {N};
-  if (M < 1 || N < 1 || ctas < 1 || !plan_gemm(M, K, 1, rws, ctas, false, &g)) return 0;
+  if (M < 1 || N < 1 || ctas < 1 || !plan_gemm(M, K, 1, rws, ctas, &g)) return 0;
   return plan_part_floats(g);
 }
 
