@@ -52,26 +52,32 @@ __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) 
 
 // ------------------------------------------------------------------ residual + RMSNorm
 // x[m] += sum of the partial slots (when pv.part != nullptr); u[m] = bf16(x / rms(x) * g);
-// optionally the unrounded normed row goes to hid. One CTA per row; every thread issues all
-// its loads at once (one trip to L2) and keeps its values in registers for the second pass;
-// the gains do not depend on the previous kernel and are fetched before the dependency wait.
-// d % 4 == 0.
-constexpr int NORM_THREADS = 1024;
+// optionally the unrounded normed row goes to hid. A cluster of NORM_CLUSTER CTAs (on
+// neighbouring SMs) shares a row, each with its own slice of the columns, so that one SM does
+// not have to pull a whole row's partial sums through its load queues; the slices' sums of
+// squares are exchanged through distributed shared memory and added in rank order. Every
+// thread issues all its loads at once (one trip to L2) and keeps its values in registers; the
+// gains do not depend on the previous kernel and are fetched before the dependency wait.
+// d % 4 == 0; grid (rows, NORM_CLUSTER).
+constexpr int NORM_THREADS = 512;
+constexpr int NORM_CLUSTER = 2;
 constexpr int NORM_CACHE = 2;   // float4 values a thread keeps between the two passes
 
-__global__ void __launch_bounds__(NORM_THREADS)
+__global__ void __cluster_dims__(1, NORM_CLUSTER, 1) __launch_bounds__(NORM_THREADS)
 norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict__ gain, float eps,
                bf16* __restrict__ u, float* __restrict__ hid, int d, unsigned long long* tr) {
   KTrace kt(tr);
   pdl_launch_dependents();
-  const int m = blockIdx.x;
+  const int m = blockIdx.x, rank = blockIdx.y;
   float* xr = x + (size_t)m * d;
   const int n4 = d >> 2;
+  const int per = (n4 + NORM_CLUSTER - 1) / NORM_CLUSTER;
+  const int c_lo = rank * per, c_hi = min(n4, c_lo + per);
   float4 gk[NORM_CACHE];
 #pragma unroll
   for (int k = 0; k < NORM_CACHE; ++k) {
-    const int c4 = threadIdx.x + k * NORM_THREADS;
-    gk[k] = c4 < n4 ? *reinterpret_cast<const float4*>(gain + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    const int c4 = c_lo + threadIdx.x + k * NORM_THREADS;
+    gk[k] = c4 < c_hi ? *reinterpret_cast<const float4*>(gain + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   pdl_wait();
   if (threadIdx.x == 0) trace_mark_min(tr, 2);
@@ -79,8 +85,8 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
   float ss = 0.f;
 #pragma unroll
   for (int k = 0; k < NORM_CACHE; ++k) {
-    const int c4 = threadIdx.x + k * NORM_THREADS;
-    if (c4 < n4) {
+    const int c4 = c_lo + threadIdx.x + k * NORM_THREADS;
+    if (c4 < c_hi) {
       float4 v = *reinterpret_cast<const float4*>(xr + c4 * 4);
       if (pv.part) {
         const float4 a = part_sum4(pv, m, c4 * 4);
@@ -91,7 +97,7 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
       ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
   }
-  for (int c4 = threadIdx.x + NORM_CACHE * NORM_THREADS; c4 < n4; c4 += NORM_THREADS) {
+  for (int c4 = c_lo + threadIdx.x + NORM_CACHE * NORM_THREADS; c4 < c_hi; c4 += NORM_THREADS) {
     float4 v = *reinterpret_cast<const float4*>(xr + c4 * 4);
     if (pv.part) {
       const float4 a = part_sum4(pv, m, c4 * 4);
@@ -101,12 +107,29 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   __shared__ float red[32];
+  __shared__ float slice_ss;
   ss = warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < (NORM_THREADS >> 5); ++w) t += red[w];
+    slice_ss = t;
+  }
+  // exchange the slices' sums through distributed shared memory (cluster barrier: release / acquire)
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
   float tot = 0.f;
 #pragma unroll
-  for (int w = 0; w < (NORM_THREADS >> 5); ++w) tot += red[w];   // same order in every thread
+  for (int r = 0; r < NORM_CLUSTER; ++r) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(&slice_ss)), "r"(r));
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    tot += v;                                           // rank order: the same sum in every CTA
+  }
+  // nobody may leave (and give up its shared memory) before every CTA has read it
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
   const float inv = rsqrtf(tot / (float)d + eps);
   auto emit = [&](int c4, const float4& v, const float4& g) {
     const float4 o = make_float4(v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
@@ -115,10 +138,10 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
   };
 #pragma unroll
   for (int k = 0; k < NORM_CACHE; ++k) {
-    const int c4 = threadIdx.x + k * NORM_THREADS;
-    if (c4 < n4) emit(c4, keep[k], gk[k]);
+    const int c4 = c_lo + threadIdx.x + k * NORM_THREADS;
+    if (c4 < c_hi) emit(c4, keep[k], gk[k]);
   }
-  for (int c4 = threadIdx.x + NORM_CACHE * NORM_THREADS; c4 < n4; c4 += NORM_THREADS)
+  for (int c4 = c_lo + threadIdx.x + NORM_CACHE * NORM_THREADS; c4 < c_hi; c4 += NORM_THREADS)
     emit(c4, *reinterpret_cast<const float4*>(xr + c4 * 4), *reinterpret_cast<const float4*>(gain + c4 * 4));
 }
 

@@ -524,7 +524,7 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, cons
   const int kp0 = (HD + 127) / 128 * 128, vp0 = kp0 + (KD + 127) / 128 * 128;   // padded columns of k and v in the QKV partials
   const int up0 = (F + 127) / 128 * 128;                                        // and of the up projection
 #define NORM_LAUNCH(pv, gain, uq, hid)                                                                   \
-  KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M), dim3(NORM_THREADS), 0, c->d_x, pv, gain, f.rms_eps, uq, hid, d)
+  KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M, NORM_CLUSTER), dim3(NORM_THREADS), 0, c->d_x, pv, gain, f.rms_eps, uq, hid, d)
   PartView pend{};              // partial sums of the previous down-projection still to be added to x
   for (int l = 0; l < f.n_layers; ++l) {
     NORM_LAUNCH(pend, c->an[l], u, (float*)nullptr);
