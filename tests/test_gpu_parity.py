@@ -210,3 +210,52 @@ def test_error_returns_and_degenerate_shapes(torch):
         tok, cnt = dec.step()
         assert int(cnt[0]) == 1
     dec.close()
+
+
+def test_timeline_and_options(torch):
+    """The device timeline lists every launch of a step in order with start <= end; tuning knobs
+    reject out-of-range values and do not change the emitted tokens."""
+    from paper_2503_14153_b200 import SpecDecoder, SpecError, build_tree, upload_weights
+    from paper_2503_14153_b200 import binding as B
+    cfg = SMALL_BF16
+    w = draw_weights(cfg)
+    dw = upload_weights(cfg, w)
+    tree = build_tree(cfg.topk, cfg.tree_nodes)
+    prompt = draw_prompt(cfg, 33)
+
+    def run(opts):
+        dec = SpecDecoder(cfg, dw, tree, 200)
+        for k, v in opts.items():
+            dec.set_option(k, v)
+        dec.prefill(prompt)
+        out = []
+        for _ in range(6):
+            tok, cnt = dec.step()
+            out.extend(int(t) for t in tok[0][: int(cnt[0])])
+        return dec, out
+
+    dec, base = run({})
+    with pytest.raises(SpecError):
+        dec.set_option(B.OPT_GEMM_CTAS, 0)
+    with pytest.raises(SpecError):
+        dec.set_option(99, 1)
+    with pytest.raises(SpecError):
+        dec.trace()                                     # tracing is off
+    dec.set_option(B.OPT_TRACE, 1)
+    l0 = dec.query(B.Q_KERNEL_LAUNCHES)
+    dec.step()
+    n_launch = dec.query(B.Q_KERNEL_LAUNCHES) - l0
+    tr = dec.trace()
+    assert len(tr) == n_launch and n_launch > 10
+    names = [r[0] for r in tr]
+    assert names[-1] == "compact_kv" and "attention_tc" in names and any(n.startswith("gemm") for n in names)
+    for name, t0, t1, _, _ in tr:
+        assert 0 < t0 <= t1, (name, t0, t1)
+    assert tr[0][1] <= tr[-1][2]
+    dec.close()
+    # programmatic dependent launch and L2 prefetch never change results; the CTA count only the
+    # summation order (same tokens here: no near-tie in these steps)
+    for opts in ({B.OPT_PDL: 0}, {B.OPT_L2_PREFETCH: 4}):
+        d2, out = run(opts)
+        d2.close()
+        assert out == base
