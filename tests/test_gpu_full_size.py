@@ -127,3 +127,70 @@ def test_c4_batch16_matches_single_sequence_runs(torch):
             assert err < TOL_BF16, (b, err)
         else:
             assert k >= 2, (b, out, emitted[b])
+
+
+def test_c2_controlled_draft_full_size(torch):
+    """Configuration 2 at full size (32 layers, 512-token prompt, T = 64): with the controlled draft the
+    emitted stream stays the plain greedy stream (lossless acceptance) up to a near tie of the base
+    model's logits (a different draft changes tree slots and tile boundaries, hence float32 summation
+    order), and the mean accepted length follows the closed form sum_i p^i within its sampling error."""
+    from paper_2503_14153_b200 import SpecDecoder, build_tree
+    from paper_2503_14153_b200 import binding as B
+    from synthetic import controlled_draft, stream_weights_to_device
+    cfg = get_config("c2")
+    dw = stream_weights_to_device(cfg, "cuda:0", threads=16)
+    tree = build_tree(cfg.topk, cfg.tree_nodes)
+    prompt = draw_prompt(cfg)
+    new_tokens = 256
+    K = cfg.n_medusa
+    dec = SpecDecoder(cfg, dw, tree, cfg.prompt_len + new_tokens + 16, flags=B.FLAG_KEEP_LOGITS)
+
+    def generate(p, stream=None, want_gaps=False):
+        dec.prefill(prompt)
+        out, counts, gaps, step = [], [], [np.inf], 0
+        uniforms, hit = (None, None) if p is None else controlled_draft(cfg, None, p, new_tokens)
+        while len(out) < new_tokens:
+            ov = None
+            if p is not None:
+                ov = uniforms[step].copy()
+                for j in range(K):
+                    pos = len(out) + 1 + j                # generated position head j predicts
+                    if hit[step, j] and pos < len(stream):
+                        ov[j, 0] = stream[pos]
+                ov = ov[None, :, :dec.kmax]               # the library keeps only the ranks the tree uses
+            tok, cnt = dec.step(ov)
+            c = int(cnt[0])
+            if want_gaps:
+                # the token after path node v is the argmax of the logits row of v
+                logits = dec.debug(B.DBG_LOGITS)
+                for v in dec.debug(B.DBG_PATH)[0][:c]:
+                    top2 = np.partition(logits[int(v)], -2)[-2:]
+                    gaps.append(float(top2[1] - top2[0]))
+            out.extend(int(t) for t in tok[0][:c])
+            counts.append(c)
+            step += 1
+        return out, counts, gaps
+
+    stream, _, gaps = generate(None, want_gaps=True)
+    stream = stream + [0] * 8
+    for p in (0.3, 0.6, 0.9):
+        out, counts, _ = generate(p, stream)
+        n = min(new_tokens, len(out))
+        k = next((i for i in range(n) if out[i] != stream[i]), n)
+        if k < n:
+            assert gaps[k] < TIE_GAP_32_LAYERS, f"p={p}: stream differs at {k} where the top-2 gap is {gaps[k]}"
+        # steps that ended before the divergence follow the draft's statistics
+        done, good = 0, []
+        for c in counts[:-1]:
+            done += c
+            if done <= k:
+                good.append(c)
+        assert k >= 32 and len(good) >= 8, (p, k, len(good))
+        want = sum(p ** i for i in range(K + 1))
+        got = float(np.mean(good))
+        # counts lie in [1, K+1]: standard error at most (K/2)/sqrt(steps); allow 4 of them
+        tol = 4 * (K / 2) / np.sqrt(len(good)) + 0.05
+        assert abs(got - want) < tol, (p, got, want, tol)
+        print(f"controlled draft p={p}: mean accepted length {got:.3f} (closed form {want:.3f}) over {len(good)} steps; "
+              f"stream identical for {k} of {n} tokens")
+    dec.close()
