@@ -138,7 +138,8 @@ const char *spec_last_error(const spec_ctx *ctx);
 
 /* Integer properties of a context. */
 enum { SPEC_Q_KMAX = 0, SPEC_Q_KERNEL_LAUNCHES = 1, SPEC_Q_N_NODES = 2, SPEC_Q_BATCH = 3,
-       SPEC_Q_ALGO_BYTES_PER_STEP = 4 /* weights + lm_head (twice) + heads, in KiB */ };
+       SPEC_Q_ALGO_BYTES_PER_STEP = 4 /* weights + lm_head (twice) + heads, in KiB */,
+       SPEC_Q_GRAPH_CAPTURES = 5 /* times a step was recorded into a CUDA graph */ };
 int64_t spec_query(const spec_ctx *ctx, int32_t what);
 
 /* Tuning knobs of a context (defaults in brackets). SPEC_OPT_PDL [1]: launch the kernels of
@@ -150,9 +151,13 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
  * chunks each GEMM CTA requests into L2, beyond its shared-memory ring, before it waits for the
  * previous kernel (0..64). Results do not depend on SPEC_OPT_PDL or SPEC_OPT_L2_PREFETCH;
  * SPEC_OPT_GEMM_CTAS and SPEC_OPT_SMALL_GEMM_CTAS change the order in which partial sums are added. SPEC_OPT_TRACE [0]:
- * record a device timeline of every step (see spec_trace_read). */
+ * record a device timeline of every step (see spec_trace_read). SPEC_OPT_GRAPH [1]: record the
+ * kernel sequence of a step into a CUDA graph once and replay it on the following steps (a new
+ * recording when a sequence grows past the 256-position bound the attention launches were planned
+ * for, after a prefill and after an option change; steps that are traced or profiled are enqueued
+ * directly). Results do not depend on it. */
 enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2, SPEC_OPT_TRACE = 3,
-       SPEC_OPT_SMALL_GEMM_CTAS = 4 };
+       SPEC_OPT_SMALL_GEMM_CTAS = 4, SPEC_OPT_GRAPH = 5 };
 int spec_set_option(spec_ctx *ctx, int32_t what, int32_t value);
 
 /* Device timeline of the LAST step, recorded while SPEC_OPT_TRACE is on: one record per kernel

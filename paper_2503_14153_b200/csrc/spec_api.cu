@@ -214,6 +214,22 @@ struct spec_ctx {
     trace_names.push_back(name);
     return d_trace + 4 * (size_t)(trace_n++);
   }
+  // CUDA-graph replay of the step's kernel sequence: one instantiated graph per (override given?)
+  // variant, valid while the sequences stay below the length bound its attention launches were
+  // planned for and no option changed (epoch)
+  bool graph_on = true;
+  bool capturing = false;
+  cudaStream_t cap_stream = nullptr;
+  struct StepGraph {
+    cudaGraphExec_t exec = nullptr;
+    unsigned long long epoch = 0;
+    int B = 0;
+    long long n_launches = 0;
+    std::vector<int> n_hi_plan, n_lo_plan;
+  };
+  StepGraph step_graph[2];
+  unsigned long long graph_epoch = 1;
+  long long graph_captures = 0;
   bool prefilled = false;
   // timing: phase boundaries of the last step; optional per-launch timing of one kernel kind
   cudaEvent_t phase_ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -709,6 +725,7 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
   }
   c->B = batch;
   c->prefilled = false;
+  c->graph_epoch++;   // recorded steps were planned for the previous sequences
   std::vector<int> off(batch + 1);
   for (int b = 0; b <= batch; ++b) off[b] = offsets[b] - offsets[0];
   CUDA_OK(cudaMemsetAsync(c->d_status, 0, 4 * sizeof(int), c->stream));
@@ -745,26 +762,19 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
   return SPEC_OK;
 }
 
+// Phase boundary i of the step: an event record (an external-event node while the step is being captured).
+void step_event(spec_ctx* c, int i) {
+  if (c->capturing) cudaEventRecordWithFlags(c->phase_ev[i], c->stream, cudaEventRecordExternal);
+  else cudaEventRecord(c->phase_ev[i], c->stream);
+}
+
+// Enqueues the kernels of one step (or records them, when the stream is capturing). ov: device
+// candidate overrides or null; n_hi_plan / n_lo_plan: the length bounds the attention launches are planned for.
 template <typename T>
-int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t* cand_override) {
+int step_body(spec_ctx* c, const int* ov, const int* n_hi_plan, const int* n_lo_plan) {
   const spec_config& f = c->cfg;
   int B = c->B, K = c->K, T_ = c->T, d = f.d_model, kmax = c->kmax;
-  for (int b = 0; b < B; ++b)
-    if (c->n_hi[b] + K + 1 > f.max_seq) return c->fail(SPEC_E_SEQLEN, "sequence would exceed max_seq");
-  for (int i = 0; i < 6; ++i)
-    if (!c->phase_ev[i]) CUDA_OK(cudaEventCreate(&c->phase_ev[i]));
-  c->prof_used = 0;
-  if (c->trace_on) {
-    c->trace_n = 0;
-    c->trace_names.clear();
-    CUDA_OK(cudaMemcpyAsync(c->d_trace, c->trace_init.data(), c->trace_init.size() * 8, cudaMemcpyHostToDevice, c->stream));
-  }
-  cudaEventRecord(c->phase_ev[0], c->stream);
-  const int* ov = nullptr;
-  if (cand_override && K > 0) {
-    CUDA_OK(cudaMemcpyAsync(c->d_cand_ov, cand_override, (size_t)B * K * kmax * sizeof(int), cudaMemcpyHostToDevice, c->stream));
-    ov = c->d_cand_ov;
-  }
+  step_event(c, 0);
   // (1) extra heads -> shared lm_head -> per-head top-k -> candidate table
   if (K > 0 && c->tc) {
     int r = heads_tc(c, ov);
@@ -786,19 +796,19 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   } else {
     CUDA_OK(cudaMemcpyAsync(c->d_cand, c->d_root, B * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
   }
-  cudaEventRecord(c->phase_ev[1], c->stream);
+  step_event(c, 1);
   // (2) candidate tree -> rows
   int M = B * T_;
   Rows rows = make_rows(c, T_, false);
   KLAUNCH("prepare_verify_rows", prepare_verify_rows<T>, dim3(M), dim3(128), 0, rows, (const int*)c->d_cand, (K + 1) * kmax, kmax,
           (const int*)c->d_depth, (const int*)c->d_rank, c->cap, static_cast<const T*>(c->embed), c->d_x, d, f.vocab, c->d_status);
-  cudaEventRecord(c->phase_ev[2], c->stream);
+  step_event(c, 2);
   // (3) verification forward
-  int r = forward_layers<T>(c, T_, false, c->n_hi.data(), c->n_lo.data());
+  int r = forward_layers<T>(c, T_, false, n_hi_plan, n_lo_plan);
   if (r) return r;
   r = lm_head_argmax<T>(c, static_cast<const T*>(c->d_hq), M);
   if (r) return r;
-  cudaEventRecord(c->phase_ev[3], c->stream);
+  step_event(c, 3);
   // (4) acceptance
   AcceptArgs a = make_accept(c, T_, 0);
   if (f.accept_mode == 1) {
@@ -808,12 +818,78 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     a.edge_ok = c->d_edge;
   }
   KLAUNCH("accept_kernel", accept_kernel, dim3(B), dim3(256), 0, a);
-  cudaEventRecord(c->phase_ev[4], c->stream);
+  step_event(c, 4);
   // (5) KV compaction
   dim3 gc(f.n_layers * 2 * f.n_kv_heads, B);
   KLAUNCH("compact_kv", compact_kv<T>, gc, dim3(64), 0, static_cast<T*>(c->d_pool), c->geom, (const int*)c->d_page_table,
           (const int*)c->d_path, (const int*)c->d_count, (const int*)c->d_n_old, K);
-  cudaEventRecord(c->phase_ev[5], c->stream);
+  step_event(c, 5);
+  return SPEC_OK;
+}
+
+template <typename T>
+int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t* cand_override) {
+  const spec_config& f = c->cfg;
+  int B = c->B, K = c->K, T_ = c->T, d = f.d_model, kmax = c->kmax;
+  for (int b = 0; b < B; ++b)
+    if (c->n_hi[b] + K + 1 > f.max_seq) return c->fail(SPEC_E_SEQLEN, "sequence would exceed max_seq");
+  for (int i = 0; i < 6; ++i)
+    if (!c->phase_ev[i]) CUDA_OK(cudaEventCreate(&c->phase_ev[i]));
+  c->prof_used = 0;
+  if (c->trace_on) {
+    c->trace_n = 0;
+    c->trace_names.clear();
+    CUDA_OK(cudaMemcpyAsync(c->d_trace, c->trace_init.data(), c->trace_init.size() * 8, cudaMemcpyHostToDevice, c->stream));
+  }
+  const int* ov = nullptr;
+  if (cand_override && K > 0) {
+    CUDA_OK(cudaMemcpyAsync(c->d_cand_ov, cand_override, (size_t)B * K * kmax * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    ov = c->d_cand_ov;
+  }
+  // the attention launches are planned for a length bound rounded up to 256 positions, so that the
+  // same launch shapes (and a captured graph) serve many steps; results do not depend on the bound
+  std::vector<int> n_hi_plan(B), n_lo_plan(B);
+  for (int b = 0; b < B; ++b) {
+    n_hi_plan[b] = std::min((int)round_up((size_t)c->n_hi[b] + T_, 256), c->cap) - T_;
+    n_lo_plan[b] = c->n_lo[b];
+  }
+  const bool use_graph = c->graph_on && !c->trace_on && c->profile_kind == 0;
+  if (!use_graph) {
+    int r = step_body<T>(c, ov, n_hi_plan.data(), n_lo_plan.data());
+    if (r) return r;
+  } else {
+    spec_ctx::StepGraph& g = c->step_graph[ov ? 1 : 0];
+    bool valid = g.exec && g.epoch == c->graph_epoch && g.B == B;
+    for (int b = 0; valid && b < B; ++b) valid = c->n_hi[b] <= g.n_hi_plan[b] && c->n_lo[b] >= g.n_lo_plan[b];
+    if (!valid) {
+      // record the step once, then replay it until a sequence outgrows the planned bound
+      cudaGraph_t graph = nullptr;
+      const long long l0 = c->launches;
+      // recorded on a stream of the library's own (the caller's may be the legacy default stream,
+      // which cannot be captured); the graph is then launched on the caller's stream
+      if (!c->cap_stream) CUDA_OK(cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
+      CUDA_OK(cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal));
+      cudaStream_t user_stream = c->stream;
+      c->stream = c->cap_stream;
+      c->capturing = true;
+      int r = step_body<T>(c, ov, n_hi_plan.data(), n_lo_plan.data());
+      c->capturing = false;
+      c->stream = user_stream;
+      cudaError_t e = cudaStreamEndCapture(c->cap_stream, &graph);
+      if (r) { if (graph) cudaGraphDestroy(graph); c->launches = l0; return r; }
+      if (e != cudaSuccess || !graph) { c->launches = l0; return c->fail(SPEC_E_CUDA, std::string("step capture: ") + cudaGetErrorString(e)); }
+      if (g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+      e = cudaGraphInstantiate(&g.exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (e != cudaSuccess) { g.exec = nullptr; c->launches = l0; return c->fail(SPEC_E_CUDA, std::string("step graph instantiate: ") + cudaGetErrorString(e)); }
+      g.epoch = c->graph_epoch; g.B = B; g.n_launches = c->launches - l0;
+      g.n_hi_plan = n_hi_plan; g.n_lo_plan = n_lo_plan;
+      c->launches = l0;
+      c->graph_captures++;
+    }
+    CUDA_OK(cudaGraphLaunch(g.exec, c->stream));
+    c->launches += g.n_launches;
+  }
   c->phase_valid = true;
   if (c->profile_kind) {
     CUDA_OK(cudaStreamSynchronize(c->stream));
@@ -827,7 +903,7 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     if (out_counts) CUDA_OK(cudaMemcpyAsync(out_counts, c->d_count, (size_t)B * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
     std::vector<int> nn(B);
     CUDA_OK(cudaMemcpyAsync(nn.data(), c->d_n, B * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
-    r = check_status(c);   // synchronises
+    int r = check_status(c);   // synchronises
     if (r) return r;
     for (int b = 0; b < B; ++b) c->n_hi[b] = c->n_lo[b] = nn[b];
     c->n_copy_pending = false;
@@ -999,6 +1075,8 @@ int spec_destroy(spec_ctx* c) {
   cudaStreamSynchronize(c->stream);
   for (int i = 0; i < 6; ++i) if (c->phase_ev[i]) cudaEventDestroy(c->phase_ev[i]);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+  for (auto& g : c->step_graph) if (g.exec) cudaGraphExecDestroy(g.exec);
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
   if (c->n_ev) cudaEventDestroy(c->n_ev);
   if (c->h_n_pinned) cudaFreeHost(c->h_n_pinned);
   delete c;
@@ -1015,6 +1093,7 @@ int64_t spec_query(const spec_ctx* c, int32_t what) {
     case SPEC_Q_KERNEL_LAUNCHES: return c->launches;
     case SPEC_Q_N_NODES: return c->T;
     case SPEC_Q_BATCH: return c->B;
+    case SPEC_Q_GRAPH_CAPTURES: return c->graph_captures;
     case SPEC_Q_ALGO_BYTES_PER_STEP: {
       double d = f.d_model, F = f.d_ffn, V = f.vocab, HD = (double)f.n_heads * f.head_dim, KD = (double)f.n_kv_heads * f.head_dim;
       double layer = d * HD + 2 * d * KD + HD * d + 3 * d * F;
@@ -1027,7 +1106,10 @@ int64_t spec_query(const spec_ctx* c, int32_t what) {
 
 int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
   if (!c) return SPEC_E_BADARG;
+  c->graph_epoch++;   // a recorded step no longer matches the options
   switch (what) {
+    case SPEC_OPT_GRAPH:
+      c->graph_on = value != 0; return SPEC_OK;
     case SPEC_OPT_PDL: c->pdl = value != 0; return SPEC_OK;
     case SPEC_OPT_GEMM_CTAS:
       if (value < 1 || value > SM_SLOTS) return c->fail(SPEC_E_BADARG, "gemm CTA count out of range");

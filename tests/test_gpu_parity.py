@@ -255,7 +255,48 @@ def test_timeline_and_options(torch):
     dec.close()
     # programmatic dependent launch and L2 prefetch never change results; the CTA count only the
     # summation order (same tokens here: no near-tie in these steps)
-    for opts in ({B.OPT_PDL: 0}, {B.OPT_L2_PREFETCH: 4}):
+    for opts in ({B.OPT_PDL: 0}, {B.OPT_L2_PREFETCH: 4}, {B.OPT_GRAPH: 0}):
         d2, out = run(opts)
         d2.close()
         assert out == base
+
+
+def test_step_graph_replay(torch):
+    """The step is recorded into a CUDA graph once and replayed: one recording serves the steps until a
+    sequence passes the 256-position bound the attention launches were planned for, then one more is made;
+    a new prefill and an option change also start a new recording; the tokens are those of direct enqueue."""
+    from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights
+    from paper_2503_14153_b200 import binding as B
+    cfg = SMALL_BF16
+    dw = upload_weights(cfg, draw_weights(cfg))
+    tree = build_tree(cfg.topk, cfg.tree_nodes)
+    prompt = draw_prompt(cfg, 200)
+
+    def run(graph, steps):
+        dec = SpecDecoder(cfg, dw, tree, 600)
+        dec.set_option(B.OPT_GRAPH, graph)
+        dec.prefill(prompt)
+        out, caps = [], []
+        for _ in range(steps):
+            tok, cnt = dec.step()
+            out.extend(int(t) for t in tok[0][: int(cnt[0])])
+            caps.append(dec.query(B.Q_GRAPH_CAPTURES))
+        return dec, out, caps
+
+    d0, direct, caps0 = run(0, 60)
+    assert caps0[-1] == 0
+    d0.close()
+    d1, replay, caps1 = run(1, 60)
+    assert replay == direct
+    # 200 prompt tokens + 16 tree rows fit the first 256-position bound for the first steps only
+    assert caps1[0] == 1 and caps1[5] == 1 and caps1[-1] == 2, caps1
+    launches = d1.query(B.Q_KERNEL_LAUNCHES)
+    d1.step()
+    assert d1.query(B.Q_KERNEL_LAUNCHES) - launches > 10        # replayed launches are counted
+    d1.set_option(B.OPT_PDL, 0)
+    d1.step()
+    assert d1.query(B.Q_GRAPH_CAPTURES) == 3
+    d1.prefill(prompt)
+    d1.step()
+    assert d1.query(B.Q_GRAPH_CAPTURES) == 4
+    d1.close()
