@@ -153,8 +153,8 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
  * SPEC_OPT_GEMM_CTAS and SPEC_OPT_SMALL_GEMM_CTAS change the order in which partial sums are added. SPEC_OPT_TRACE [0]:
  * record a device timeline of every step (see spec_trace_read). SPEC_OPT_GRAPH [1]: record the
  * kernel sequence of a step into a CUDA graph once and replay it on the following steps (a new
- * recording when a sequence grows past the 256-position bound the attention launches were planned
- * for, after a prefill and after an option change; steps that are traced or profiled are enqueued
+ * recording when a sequence grows past the 768 positions the single-split attention launch covers,
+ * after a prefill and after an option change; steps that are traced or profiled are enqueued
  * directly). Results do not depend on it. */
 enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2, SPEC_OPT_TRACE = 3,
        SPEC_OPT_SMALL_GEMM_CTAS = 4, SPEC_OPT_GRAPH = 5 };

@@ -7,10 +7,13 @@
 // copies that complete on an mbarrier (the cache's in-page chunk swizzle makes the landed
 // tile conflict-free for ldmatrix); QK^T and PV run on mma.sync m16n8k16 with a warp-level
 // online softmax; the tree mask is a 128-bit ancestor set per row applied only to keys at or
-// beyond the committed length. The host picks the number of KV splits from its bound on the
-// context length; tiles that hold only rows of earlier steps are fetched before the wait on
-// the previous kernel. With one split the CTA writes the normalised bf16 output
-// itself, otherwise each split leaves (max, sum, unnormalised output) and the CTA of a
+// beyond the committed length. The host only picks the launch shape (one CTA per head and 16-row
+// block for short contexts, or up to `nsplit` KV splits per head) from its bound on the context
+// length; how many of the launched splits are used, and the tiles of each, follow from the
+// sequence length on the device, so one launch shape (and a recorded graph) serves a whole
+// range of lengths. With a single split, tiles that hold only rows of earlier steps are
+// fetched before the wait on the previous kernel and the CTA writes the normalised bf16 output
+// itself; otherwise each split leaves (max, sum, unnormalised output) and the CTA of a
 // (sequence, head) that finishes last (arrival counter, no waiting) merges them.
 #pragma once
 #include "common.cuh"
@@ -50,8 +53,7 @@ struct AttnTcArgs {
   const int* page_table;
   Rows rows;
   int layer, H;
-  int nsplit;           // KV splits (= gridDim.y), chosen by the host from its bound on the context length
-  int tps;              // KV tiles per split
+  int nsplit;           // KV splits launched (gridDim.y = nsplit * row_blocks); the splits in use are min(nsplit, ceil(tiles / 8))
   int stages;           // KV tiles in flight per CTA (2..ATTN_MAX_STAGES, at least KG); sizes the shared memory
   int row_blocks;       // CTAs that share a (head, split): CTA j of them owns query rows [16 NW j, 16 NW (j+1)); > 1 only with nsplit == 1
   int n_lo[ATTN_MAX_SEQS];   // host's lower bound of each sequence's committed length: keys below it
@@ -104,19 +106,17 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   const int h = blockIdx.x, sp = blockIdx.y / a.row_blocks, b = blockIdx.z;
   const int row0 = (blockIdx.y % a.row_blocks) * NW * 16;        // first query row of this CTA
   const int H = a.H, kvh = h / (H / a.g.n_kv_heads);
-  const int nsplit = a.nsplit, tps = a.tps;
-  const int t0 = sp * tps;
+  const bool single = a.nsplit == 1;          // one split: its tiles start at 0 whatever the length
   const int* pt = a.page_table + b * a.g.pages_per_seq;
   if (threadIdx.x == 0) {
     for (int i = 0; i < ST; ++i) mbar_init(&full[i], 1);
     mbar_fence_init();
   }
-  // the page table is fixed at set-up: stage this split's entries before the dependency wait
-  for (int e = threadIdx.x; e < tps * (KT / 16) && e < ATTN_PT_CACHE; e += NTHR) {
-    const int idx = t0 * (KT / 16) + e;
-    pt_s[e] = idx < a.g.pages_per_seq ? pt[idx] : 0;
-  }
+  // the page table is fixed at set-up: with a single split its first entries are staged before the dependency wait
+  if (single)
+    for (int e = threadIdx.x; e < ATTN_PT_CACHE; e += NTHR) pt_s[e] = e < a.g.pages_per_seq ? pt[e] : 0;
   __syncthreads();   // barriers initialised, page entries staged
+  int t0 = 0;
   auto issue = [&](int tile, int buf) {
     mbar_expect_tx(&full[buf], 2 * TILE_BYTES);
     for (int pg = 0; pg < KT / 16; ++pg) {
@@ -131,10 +131,9 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   // tiles that lie wholly below the host's lower bound of the committed length hold rows of
   // earlier steps: start fetching them now (thread 0 keeps the count)
   int pre = 0;
-  if (threadIdx.x == 0) {
+  if (single && threadIdx.x == 0) {
     const int safe = (b < ATTN_MAX_SEQS ? a.n_lo[b] : 0) / KT;      // tiles [0, safe) are committed
-    const int lim = min(t0 + tps, safe);
-    for (; pre < ST && t0 + pre < lim; ++pre) issue(t0 + pre, pre);
+    for (; pre < ST && pre < safe; ++pre) issue(pre, pre);
   }
   pdl_wait();
   if (threadIdx.x == 0) trace_mark_min(tr, 2);
@@ -157,12 +156,23 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   const int S = n + cnt;
   const int M = a.rows.B * R;
   const int total_tiles = (S + KT - 1) / KT;
+  // the splits in use and their tiles follow from the length: eight tiles or more per split
+  const int nsplit = single ? 1 : max(1, min(a.nsplit, (total_tiles + 7) / 8));
+  const int tps = (total_tiles + nsplit - 1) / nsplit;
+  t0 = sp * tps;
   const int t1 = min(total_tiles, t0 + tps);
-  if (cnt == 0) {
-    // inactive sequence: let the copies already in flight land before the CTA goes away
+  if (cnt == 0 || sp >= nsplit) {
+    // inactive sequence or unused split: let the copies already in flight land before the CTA goes away
     if (threadIdx.x == 0)
       for (int i = 0; i < pre; ++i) mbar_wait(&full[i], 0, a.status, 21);
     return;
+  }
+  if (!single) {
+    for (int e = threadIdx.x; e < tps * (KT / 16) && e < ATTN_PT_CACHE; e += NTHR) {
+      const int idx = t0 * (KT / 16) + e;
+      pt_s[e] = idx < a.g.pages_per_seq ? pt[idx] : 0;
+    }
+    __syncthreads();
   }
   // the rest of the first tiles
   if (threadIdx.x == 0)

@@ -32,6 +32,8 @@ thread_local std::string g_create_error = "no error";
 constexpr int PREFILL_ROWS = 128;   // rows per sequence in one prefill pass
 constexpr int TRACE_CAP = 1024;     // launches of one step the timeline can hold
 constexpr int SM_SLOTS = 296;       // 148 SMs x 2 co-resident GEMM CTAs
+constexpr int MAX_STEPS_AHEAD = 8;      // enqueue-only steps the host may run ahead of the device
+constexpr int ATTN_SINGLE_TILES = 12;   // contexts of at most this many 64-key tiles use one KV split
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -493,12 +495,11 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
     tiles_hi = std::max(tiles_hi, (n_hi_pass[b] + R + 63) / 64);
     if (b < ATTN_MAX_SEQS) a.n_lo[b] = n_lo_pass ? n_lo_pass[b] : 0;
   }
-  // short contexts: one CTA per (sequence, head) walks all tiles (no merge step); longer ones are cut
-  // into at most one split per resident CTA slot, eight tiles or more each
+  // short contexts (host bound of at most ATTN_SINGLE_TILES tiles): one split, no merge step; longer
+  // ones get as many split CTAs as fit beside each other, and the kernel uses min(that, tiles / 8) of them
   const int slots1 = std::max(1, std::min(c->nsplit_attn, (SM_SLOTS / 2) / (H * c->B)));
-  a.nsplit = tiles_hi <= 12 ? 1 : std::min(slots1, (tiles_hi + 7) / 8);
+  a.nsplit = tiles_hi <= ATTN_SINGLE_TILES ? 1 : slots1;
   a.stages = 4;
-  a.tps = (tiles_hi + a.nsplit - 1) / a.nsplit;
   a.row_blocks = 1;
   int nw = (R + 15) / 16;
   // short context and few sequences: a CTA per 16 query rows, its six warps taking a KV tile each,
@@ -846,11 +847,12 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     CUDA_OK(cudaMemcpyAsync(c->d_cand_ov, cand_override, (size_t)B * K * kmax * sizeof(int), cudaMemcpyHostToDevice, c->stream));
     ov = c->d_cand_ov;
   }
-  // the attention launches are planned for a length bound rounded up to 256 positions, so that the
-  // same launch shapes (and a captured graph) serve many steps; results do not depend on the bound
+  // the attention launch shape depends only on whether the context fits ATTN_SINGLE_TILES tiles (the
+  // kernel takes the lengths themselves from the device), so the launches are planned for one of two
+  // length bounds and a recorded step serves every length below its bound
   std::vector<int> n_hi_plan(B), n_lo_plan(B);
   for (int b = 0; b < B; ++b) {
-    n_hi_plan[b] = std::min((int)round_up((size_t)c->n_hi[b] + T_, 256), c->cap) - T_;
+    n_hi_plan[b] = (c->n_hi[b] + T_ <= ATTN_SINGLE_TILES * 64 ? std::min(ATTN_SINGLE_TILES * 64, c->cap) : c->cap) - T_;
     n_lo_plan[b] = c->n_lo[b];
   }
   const bool use_graph = c->graph_on && !c->trace_on && c->profile_kind == 0;
@@ -912,6 +914,8 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     if (c->h_n_pinned && c->n_ev) {
       if (c->n_copy_pending) {
         c->n_copy_steps_after++;
+        // the host stays at most MAX_STEPS_AHEAD steps ahead of the device, so that its bounds stay close
+        if (c->n_copy_steps_after >= MAX_STEPS_AHEAD) cudaEventSynchronize(c->n_ev);
         if (cudaEventQuery(c->n_ev) == cudaSuccess) {
           // the copy shows the lengths after an earlier step; every step since added 1..K+1 tokens
           for (int b = 0; b < B; ++b) {

@@ -263,17 +263,18 @@ def test_timeline_and_options(torch):
 
 def test_step_graph_replay(torch):
     """The step is recorded into a CUDA graph once and replayed: one recording serves the steps until a
-    sequence passes the 256-position bound the attention launches were planned for, then one more is made;
-    a new prefill and an option change also start a new recording; the tokens are those of direct enqueue."""
+    sequence passes the 768-position bound of the single-split attention launch, then one more is made
+    (for every longer length); a new prefill and an option change also start a new recording; the
+    tokens are those of direct enqueue."""
     from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights
     from paper_2503_14153_b200 import binding as B
     cfg = SMALL_BF16
     dw = upload_weights(cfg, draw_weights(cfg))
     tree = build_tree(cfg.topk, cfg.tree_nodes)
-    prompt = draw_prompt(cfg, 200)
+    prompt = draw_prompt(cfg, 700)
 
     def run(graph, steps):
-        dec = SpecDecoder(cfg, dw, tree, 600)
+        dec = SpecDecoder(cfg, dw, tree, 1100)
         dec.set_option(B.OPT_GRAPH, graph)
         dec.prefill(prompt)
         out, caps = [], []
@@ -288,7 +289,7 @@ def test_step_graph_replay(torch):
     d0.close()
     d1, replay, caps1 = run(1, 60)
     assert replay == direct
-    # 200 prompt tokens + 16 tree rows fit the first 256-position bound for the first steps only
+    # 700 prompt tokens + 16 tree rows fit the 768-position bound for the first steps only
     assert caps1[0] == 1 and caps1[5] == 1 and caps1[-1] == 2, caps1
     launches = d1.query(B.Q_KERNEL_LAUNCHES)
     d1.step()
