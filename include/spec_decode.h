@@ -13,8 +13,10 @@
  *    throws or traps; spec_last_error() gives a one-line description of the last failure.
  *  - "DEVICE" pointers are CUDA global memory of the device that was current at
  *    spec_create. "HOST" pointers are ordinary (preferably pinned) host memory.
- *  - The library never allocates or frees device memory. The caller owns weights,
- *    workspace and the stream; they must outlive the context.
+ *  - The library never calls the device allocator: every buffer it uses lies in the
+ *    caller's workspace. (With SPEC_OPT_GRAPH the CUDA runtime keeps an instantiated graph
+ *    of the step and the library one extra stream to record it on.) The caller owns
+ *    weights, workspace and the stream; they must outlive the context.
  *  - Linear weights are row-major [out_features, in_features]; dtype 0 = float32,
  *    dtype 1 = bfloat16 (operands bf16, accumulation and residual stream float32).
  */

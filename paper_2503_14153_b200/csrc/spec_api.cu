@@ -1,6 +1,7 @@
 // C ABI of the draft-and-verify decode loop: context set-up, workspace carving, the
 // per-step kernel schedule and the debug taps. All device work is enqueued on the caller's
-// stream; the library allocates no device memory.
+// stream (a step is recorded once on a stream of the library's own and replayed on the caller's);
+// every device buffer lies in the caller's workspace.
 #include "../../include/spec_decode.h"
 
 #include <cuda.h>
