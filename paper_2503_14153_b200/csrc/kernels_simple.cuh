@@ -476,11 +476,31 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptArgs a, unsigned long
   }
   __syncthreads();
   if (len_s > 0) {
-    const float* src = a.hid + (size_t)(m0 + last_s) * a.d;
-    for (int c = threadIdx.x; c < a.d; c += blockDim.x) {
-      const float v = src[c];
-      a.h_last[(size_t)b * a.d + c] = v;
-      if (a.hq_last) a.hq_last[(size_t)b * a.d + c] = __float2bfloat16_rn(v);
+    // the accepted node's hidden row feeds the next step's heads (d % 4 == 0); four groups per
+    // thread are loaded before the first store, so the copy is one trip to L2 for most widths
+    const float4* src = reinterpret_cast<const float4*>(a.hid + (size_t)(m0 + last_s) * a.d);
+    float4* dst = reinterpret_cast<float4*>(a.h_last + (size_t)b * a.d);
+    const int n4 = a.d >> 2;
+    for (int c0 = threadIdx.x; c0 < n4; c0 += 4 * blockDim.x) {
+      float4 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int c = c0 + k * blockDim.x;
+        v[k] = c < n4 ? src[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int c = c0 + k * blockDim.x;
+        if (c >= n4) continue;
+        dst[c] = v[k];
+        if (a.hq_last) {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(v[k].x, v[k].y), hi = __floats2bfloat162_rn(v[k].z, v[k].w);
+          uint2 pk;
+          pk.x = *reinterpret_cast<uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(a.hq_last + (size_t)b * a.d + c * 4) = pk;
+        }
+      }
     }
   }
 }
