@@ -7,9 +7,11 @@
 // copies that complete on an mbarrier (the cache's in-page chunk swizzle makes the landed
 // tile conflict-free for ldmatrix); QK^T and PV run on mma.sync m16n8k16 with a warp-level
 // online softmax; the tree mask is a 128-bit ancestor set per row applied only to keys at or
-// beyond the committed length. The host only picks the launch shape (one CTA per head and 16-row
-// block for short contexts, or up to `nsplit` KV splits per head) from its bound on the context
-// length; how many of the launched splits are used, and the tiles of each, follow from the
+// beyond the committed length. Two kernels: attention_rows (at the end of this file) when the
+// (sequence, head, 16-row block) CTAs of the pass fit the SMs, attention_tc otherwise. For
+// attention_tc the host only picks the launch shape (one split per head for short contexts, or
+// up to `nsplit` KV splits per head) from its bound on the context length; how many of the
+// launched splits are used, and the tiles of each, follow from the
 // sequence length on the device, so one launch shape (and a recorded graph) serves a whole
 // range of lengths. With a single split, tiles that hold only rows of earlier steps are
 // fetched before the wait on the previous kernel and the CTA writes the normalised bf16 output
@@ -53,9 +55,9 @@ struct AttnTcArgs {
   const int* page_table;
   Rows rows;
   int layer, H;
-  int nsplit;           // KV splits launched (gridDim.y = nsplit * row_blocks); the splits in use are min(nsplit, ceil(tiles / 8))
+  int nsplit;           // KV splits launched (gridDim.y); the splits in use are min(nsplit, ceil(tiles / split_tiles))
+  int split_tiles;      // fewest KV tiles worth a split of their own
   int stages;           // KV tiles in flight per CTA (2..ATTN_MAX_STAGES, at least KG); sizes the shared memory
-  int row_blocks;       // CTAs that share a (head, split): CTA j of them owns query rows [16 NW j, 16 NW (j+1)); > 1 only with nsplit == 1
   int n_lo[ATTN_MAX_SEQS];   // host's lower bound of each sequence's committed length: keys below it
                              // were written by earlier steps and may be fetched before the dependency wait
   float scale_log2;     // log2(e) / sqrt(head_dim)
@@ -103,8 +105,8 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rg = warp % NW, kg = warp / NW;
-  const int h = blockIdx.x, sp = blockIdx.y / a.row_blocks, b = blockIdx.z;
-  const int row0 = (blockIdx.y % a.row_blocks) * NW * 16;        // first query row of this CTA
+  const int h = blockIdx.x, sp = blockIdx.y, b = blockIdx.z;
+  constexpr int row0 = 0;                                        // the CTA owns all query rows of its sequence
   const int H = a.H, kvh = h / (H / a.g.n_kv_heads);
   const bool single = a.nsplit == 1;          // one split: its tiles start at 0 whatever the length
   const int* pt = a.page_table + b * a.g.pages_per_seq;
@@ -156,8 +158,8 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   const int S = n + cnt;
   const int M = a.rows.B * R;
   const int total_tiles = (S + KT - 1) / KT;
-  // the splits in use and their tiles follow from the length: eight tiles or more per split
-  const int nsplit = single ? 1 : max(1, min(a.nsplit, (total_tiles + 7) / 8));
+  // the splits in use and their tiles follow from the length: split_tiles tiles or more per split
+  const int nsplit = single ? 1 : max(1, min(a.nsplit, (total_tiles + a.split_tiles - 1) / a.split_tiles));
   const int tps = (total_tiles + nsplit - 1) / nsplit;
   t0 = sp * tps;
   const int t1 = min(total_tiles, t0 + tps);
@@ -453,6 +455,282 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
         *reinterpret_cast<uint2*>(dst + e * 4) = pk;
       }
     }
+  }
+}
+
+// ------------------------------------------------------------------ one CTA per (head, 16 query rows)
+// The same attention for passes whose (sequence, head, 16-row block) count fits the GPU's SMs: a
+// CTA owns 16 query rows of one head and walks the whole context, so there is nothing to merge
+// across CTAs and the launch does not depend on the context length at all. Each of the W warps
+// streams its own sub-tiles of 32 keys (two cache pages; sub-tile w, w + W, ...) through two
+// private buffers: it waits for a buffer, works on it (QK^T, mask, online softmax, PV) and asks
+// for its next-but-one sub-tile into the same buffer, without any CTA-wide barrier in the
+// loop. The warps' softmax states are merged through shared memory at the end and warp 0
+// writes the normalised bf16 rows. Sub-tiles below the host's lower bound of the committed
+// length are requested before the wait on the previous kernel.
+__host__ __device__ inline size_t attention_rows_smem(int head_dim, int warps) {
+  const size_t rowb = (size_t)head_dim * 2;
+  return 16 * rowb + (size_t)warps * 2 * 2 * 32 * rowb + 8 * (size_t)warps * 2 + 4 * ATTN_PT_CACHE;
+}
+
+template <int HD, int W>
+__global__ void __launch_bounds__(W * 32)
+attention_rows(const AttnTcArgs a, unsigned long long* tr) {
+  KTrace kt(tr);
+  constexpr int SK = 32;                      // keys per sub-tile
+  constexpr int NB = 2;                       // buffers per warp
+  constexpr int ROWB = HD * 2;                // bytes per row
+  constexpr int SUB_BYTES = SK * ROWB;        // one operand of a sub-tile
+  constexpr int PAGE_BYTES = 16 * ROWB;
+  constexpr int NTHR = W * 32;
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* qs = smem;                                                        // [16][HD]
+  uint8_t* kv = qs + 16 * ROWB;                                              // [W][NB][K | V][SK][HD]
+  uint64_t* full = reinterpret_cast<uint64_t*>(kv + W * NB * 2 * SUB_BYTES); // [W][NB]
+  int* pt_s = reinterpret_cast<int*>(full + W * NB);                         // [ATTN_PT_CACHE]
+
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int h = blockIdx.x, b = blockIdx.z, row0 = blockIdx.y * 16;
+  const int H = a.H, kvh = h / (H / a.g.n_kv_heads);
+  const int* pt = a.page_table + b * a.g.pages_per_seq;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < W * NB; ++i) mbar_init(&full[i], 1);
+    mbar_fence_init();
+  }
+  for (int e = threadIdx.x; e < ATTN_PT_CACHE; e += NTHR) pt_s[e] = e < a.g.pages_per_seq ? pt[e] : 0;
+  __syncthreads();   // barriers initialised, page entries staged
+  uint8_t* mine = kv + (size_t)warp * NB * 2 * SUB_BYTES;
+  uint64_t* my_full = full + warp * NB;
+  auto issue = [&](int st, int bf) {          // lane 0: sub-tile st of this sequence into buffer bf
+    mbar_expect_tx(&my_full[bf], 2 * SUB_BYTES);
+#pragma unroll
+    for (int pg = 0; pg < SK / 16; ++pg) {
+      const int e = st * (SK / 16) + pg;
+      const int page = e < ATTN_PT_CACHE ? pt_s[e] : pt[e];
+      bulk_load_1d(mine + bf * 2 * SUB_BYTES + pg * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 0, kvh), PAGE_BYTES, &my_full[bf]);
+      bulk_load_1d(mine + bf * 2 * SUB_BYTES + SUB_BYTES + pg * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 1, kvh), PAGE_BYTES, &my_full[bf]);
+    }
+  };
+  // own sub-tiles that lie wholly below the host's lower bound hold rows of earlier steps
+  int issued = 0;                             // own sub-tiles requested so far (same in every lane)
+  {
+    const int safe = (b < ATTN_MAX_SEQS ? a.n_lo[b] : 0) / SK;
+    while (issued < NB && warp + issued * W < safe) {
+      if (lane == 0) issue(warp + issued * W, issued);
+      ++issued;
+    }
+  }
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  const int R = a.rows.R, cnt = a.rows.cnt[b], n = a.rows.n[b];
+  const int i0 = row0 + (lane >> 2), i1 = i0 + 8;          // this thread's two query rows
+  uint32_t anc0[4], anc1[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) { anc0[w] = a.rows.anc[i0 * 4 + w]; anc1[w] = a.rows.anc[i1 * 4 + w]; }
+  constexpr int QC = 16 * (HD / 8);                          // 16-byte chunks of the Q tile
+  constexpr int PER = (QC + NTHR - 1) / NTHR;
+  uint4 qv[PER];
+#pragma unroll
+  for (int k = 0; k < PER; ++k) {
+    const int c = threadIdx.x + k * NTHR;
+    const int r = c / (HD / 8), ch = c % (HD / 8);
+    qv[k] = make_uint4(0, 0, 0, 0);
+    if (c < QC && row0 + r < R) qv[k] = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + row0 + r) * H * HD + h * HD + ch * 8);
+  }
+  const int S = n + cnt;
+  const int n_sub = (S + SK - 1) / SK;
+  if (row0 >= cnt) {
+    // no valid row in this block: let the copies already in flight land before the CTA goes away
+    if (lane == 0)
+      for (int i = 0; i < issued; ++i) mbar_wait(&my_full[i], 0, a.status, 21);
+    return;
+  }
+  while (issued < NB && warp + issued * W < n_sub) {
+    if (lane == 0) issue(warp + issued * W, issued);
+    ++issued;
+  }
+  if (i0 >= cnt) anc0[0] = anc0[1] = anc0[2] = anc0[3] = 0u;
+  if (i1 >= cnt) anc1[0] = anc1[1] = anc1[2] = anc1[3] = 0u;
+#pragma unroll
+  for (int k = 0; k < PER; ++k) {
+    const int c = threadIdx.x + k * NTHR;
+    const int r = c / (HD / 8), ch = c % (HD / 8);
+    if (c < QC) *reinterpret_cast<uint4*>(qs + r * ROWB + ((ch ^ (r & 7)) << 4)) = (row0 + r < cnt) ? qv[k] : make_uint4(0, 0, 0, 0);
+  }
+  __syncthreads();
+  uint32_t qf[HD / 16][4];
+  {
+    const int row = (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+    for (int kk = 0; kk < HD / 16; ++kk) {
+      const int ch = kk * 2 + (lane >> 4);
+      ldmatrix_x4(smem_u32(qs + row * ROWB + ((ch ^ (row & 7)) << 4)), qf[kk]);
+    }
+  }
+  float o[HD / 8][4];
+#pragma unroll
+  for (int d = 0; d < HD / 8; ++d) o[d][0] = o[d][1] = o[d][2] = o[d][3] = 0.f;
+  float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
+
+  bool ok = true;
+  int k = 0;                                   // own sub-tiles done
+  for (int st = warp; st < n_sub; st += W, ++k) {
+    const int bf = k % NB;
+    if (!mbar_wait(&my_full[bf], (k / NB) & 1, a.status, 20)) { ok = false; break; }
+    if (st == 0 && lane == 0) trace_mark_max(tr, 3);
+    const uint8_t* kt = mine + bf * 2 * SUB_BYTES;
+    const uint8_t* vt = kt + SUB_BYTES;
+    float s[SK / 8][4];
+#pragma unroll
+    for (int j = 0; j < SK / 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+    {
+      // K fragments of a 16-wide slice of the head dimension, one slice ahead of the MMAs that use them
+      uint32_t kf[2][SK / 16][4];
+      auto load_k = [&](int kk, uint32_t (&dst)[SK / 16][4]) {
+#pragma unroll
+        for (int j2 = 0; j2 < SK / 16; ++j2) {
+          const int key = j2 * 16 + (lane & 7) + (lane >> 4) * 8;
+          const int ch = kk * 2 + ((lane >> 3) & 1);
+          ldmatrix_x4(smem_u32(kt + key * ROWB + ((ch ^ (key & 7)) << 4)), dst[j2]);
+        }
+      };
+      load_k(0, kf[0]);
+#pragma unroll
+      for (int kk = 0; kk < HD / 16; ++kk) {
+        if (kk + 1 < HD / 16) load_k(kk + 1, kf[(kk + 1) & 1]);
+#pragma unroll
+        for (int j2 = 0; j2 < SK / 16; ++j2) {
+          mma_bf16_16816(s[2 * j2], qf[kk], kf[kk & 1][j2][0], kf[kk & 1][j2][1]);
+          mma_bf16_16816(s[2 * j2 + 1], qf[kk], kf[kk & 1][j2][2], kf[kk & 1][j2][3]);
+        }
+      }
+    }
+    // mask + online softmax (log2 domain)
+    const int k0 = st * SK;
+    uint32_t vis0 = ~0u, vis1 = ~0u;
+    if (k0 + SK > n) { vis0 = (uint32_t)attn_vis64(anc0, k0, n); vis1 = (uint32_t)attn_vis64(anc1, k0, n); }
+    float tmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int j = 0; j < SK / 8; ++j) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float v = s[j][e] * a.scale_log2;
+        const int bi = j * 8 + (lane & 3) * 2 + (e & 1);
+        if (!(((e < 2 ? vis0 : vis1) >> bi) & 1u)) v = -INFINITY;
+        s[j][e] = v;
+        tmax[e >> 1] = fmaxf(tmax[e >> 1], v);
+      }
+    }
+    float alpha[2], mnew[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 1));
+      tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 2));
+      mnew[r] = fmaxf(mrow[r], tmax[r]);
+      const float base = (mnew[r] == -INFINITY) ? 0.f : mnew[r];
+      alpha[r] = exp2f(mrow[r] - base);
+      mrow[r] = mnew[r];
+      mnew[r] = base;
+      lrow[r] *= alpha[r];
+    }
+#pragma unroll
+    for (int d = 0; d < HD / 8; ++d) { o[d][0] *= alpha[0]; o[d][1] *= alpha[0]; o[d][2] *= alpha[1]; o[d][3] *= alpha[1]; }
+    uint32_t pf[SK / 16][4];
+#pragma unroll
+    for (int j = 0; j < SK / 8; ++j) {
+      const float p0 = exp2f(s[j][0] - mnew[0]), p1 = exp2f(s[j][1] - mnew[0]);
+      const float p2 = exp2f(s[j][2] - mnew[1]), p3 = exp2f(s[j][3] - mnew[1]);
+      lrow[0] += p0 + p1;
+      lrow[1] += p2 + p3;
+      pf[j >> 1][(j & 1) * 2 + 0] = pack_bf16(p0, p1);
+      pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+    {
+      // V fragments: four 16-wide slices of the head dimension at a time, one group ahead
+      constexpr int DG = 4, NG = (SK / 16) * (HD / 16) / DG;
+      uint32_t vf[2][DG][4];
+      auto load_v = [&](int g, uint32_t (&dst)[DG][4]) {
+        const int j = g / (HD / 16 / DG), d0 = (g % (HD / 16 / DG)) * DG;
+#pragma unroll
+        for (int dd = 0; dd < DG; ++dd) {
+          const int key = j * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          const int ch = (d0 + dd) * 2 + (lane >> 4);
+          ldmatrix_x4_trans(smem_u32(vt + key * ROWB + ((ch ^ (key & 7)) << 4)), dst[dd]);
+        }
+      };
+      load_v(0, vf[0]);
+#pragma unroll
+      for (int g = 0; g < NG; ++g) {
+        if (g + 1 < NG) load_v(g + 1, vf[(g + 1) & 1]);
+        const int j = g / (HD / 16 / DG), d0 = (g % (HD / 16 / DG)) * DG;
+#pragma unroll
+        for (int dd = 0; dd < DG; ++dd) {
+          mma_bf16_16816(o[2 * (d0 + dd)], pf[j], vf[g & 1][dd][0], vf[g & 1][dd][1]);
+          mma_bf16_16816(o[2 * (d0 + dd) + 1], pf[j], vf[g & 1][dd][2], vf[g & 1][dd][3]);
+        }
+      }
+    }
+    __syncwarp();                              // every lane has read the buffer: it may be refilled
+    const int nxt = st + NB * W;
+    if (nxt < n_sub && lane == 0) issue(nxt, bf);
+  }
+  if (!ok && lane == 0) {
+    // a wait gave up: the other copy this warp may still have in flight gets a bounded time to land
+    const int st1 = warp + (k + 1) * W;
+    if (st1 < n_sub) mbar_wait(&my_full[(k + 1) % NB], ((k + 1) / NB) & 1, a.status, 22);
+  }
+  ok = __syncthreads_and(ok);                  // all warps are done with their buffers
+  if (!ok) return;
+
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
+  }
+  // merge the warps' states through the (now idle) KV buffers: warps 1.. leave theirs, warp 0 adds
+  // them in warp order
+  float* ex = reinterpret_cast<float*>(kv);
+  constexpr int SLOT = (HD / 2 + 4) * 32;       // floats per warp state
+  if (warp > 0) {
+    float* my = ex + (size_t)(warp - 1) * SLOT;
+#pragma unroll
+    for (int d = 0; d < HD / 8; ++d)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) my[(d * 4 + e) * 32 + lane] = o[d][e];
+    my[(HD / 2 + 0) * 32 + lane] = mrow[0]; my[(HD / 2 + 1) * 32 + lane] = mrow[1];
+    my[(HD / 2 + 2) * 32 + lane] = lrow[0]; my[(HD / 2 + 3) * 32 + lane] = lrow[1];
+  }
+  __syncthreads();
+  if (warp != 0) return;
+#pragma unroll 1
+  for (int g2 = 1; g2 < W; ++g2) {
+    const float* th = ex + (size_t)(g2 - 1) * SLOT;
+    float w0[2], w1[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const float m1 = th[(HD / 2 + r) * 32 + lane], l1 = th[(HD / 2 + 2 + r) * 32 + lane];
+      const float mm = fmaxf(mrow[r], m1);
+      const float base = (mm == -INFINITY) ? 0.f : mm;
+      w0[r] = exp2f(mrow[r] - base);
+      w1[r] = exp2f(m1 - base);
+      mrow[r] = mm;
+      lrow[r] = lrow[r] * w0[r] + l1 * w1[r];
+    }
+#pragma unroll
+    for (int d = 0; d < HD / 8; ++d)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[d][e] = o[d][e] * w0[e >> 1] + th[(d * 4 + e) * 32 + lane] * w1[e >> 1];
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int i = r ? i1 : i0;
+    if (i >= cnt) continue;
+    const float inv = 1.f / lrow[r];
+    bf16* po = a.out + ((size_t)b * R + i) * H * HD + h * HD;
+#pragma unroll
+    for (int d = 0; d < HD / 8; ++d)
+      *reinterpret_cast<uint32_t*>(po + d * 8 + (lane & 3) * 2) = pack_bf16(o[d][2 * r] * inv, o[d][2 * r + 1] * inv);
   }
 }
 

@@ -34,6 +34,7 @@ constexpr int PREFILL_ROWS = 128;   // rows per sequence in one prefill pass
 constexpr int TRACE_CAP = 1024;     // launches of one step the timeline can hold
 constexpr int SM_SLOTS = 296;       // 148 SMs x 2 co-resident GEMM CTAs
 constexpr int MAX_STEPS_AHEAD = 8;      // enqueue-only steps the host may run ahead of the device
+constexpr int ATTN_ROWS_WARPS = 6;      // warps of the CTA-per-16-rows attention kernel
 constexpr int ATTN_SINGLE_TILES = 12;   // contexts of at most this many 64-key tiles use one KV split
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -183,6 +184,8 @@ struct spec_ctx {
   bool pdl = true;                     // programmatic dependent launch between the kernels of a step
   int gemm_ctas = 288;                 // persistent CTAs of the weight-streaming GEMM (measured best; at most SM_SLOTS)
   int l2_prefetch = 0;
+  int attn_split_tiles = 8;            // fewest KV tiles a split of the attention gets
+  int attn_single_tiles = ATTN_SINGLE_TILES;
   int small_gemm_ctas = 192;           // CTAs of GEMMs with at most 48 weight tiles (Wo, down): fewer partial sums                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
   std::vector<int> h_parent, h_depth, h_rank;
   std::vector<int> n_hi, n_lo;         // host upper / lower bounds of the committed lengths
@@ -480,6 +483,13 @@ int linear_simple(spec_ctx* c, const T* x, int ldx, const T* W, float* y, int ld
     if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string(name) + ": " + cudaGetErrorString(e_)); \
   } while (0)
 
+// Passes with several 16-row blocks whose (sequence, head, row block) CTAs fit the SMs in one wave
+// use the kernel that needs no merge across CTAs and no length-dependent launch shape.
+bool attn_rows_mode(const spec_ctx* c, int R) {
+  const int nw = (R + 15) / 16;
+  return nw > 1 && c->cfg.n_heads * c->B * nw <= SM_SLOTS / 2;
+}
+
 // n_hi_pass / n_lo_pass: host bounds of the cached length the pass's rows sit on, per sequence
 // (n_lo_pass may be null: nothing is fetched before the dependency wait).
 int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* n_hi_pass, const int* n_lo_pass) {
@@ -496,18 +506,31 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
     tiles_hi = std::max(tiles_hi, (n_hi_pass[b] + R + 63) / 64);
     if (b < ATTN_MAX_SEQS) a.n_lo[b] = n_lo_pass ? n_lo_pass[b] : 0;
   }
-  // short contexts (host bound of at most ATTN_SINGLE_TILES tiles): one split, no merge step; longer
-  // ones get as many split CTAs as fit beside each other, and the kernel uses min(that, tiles / 8) of them
+  const int nw = (R + 15) / 16;
+  if (attn_rows_mode(c, R)) {
+    // few sequences: a CTA per (head, 16 query rows) walks the whole context, whatever its length
+    a.nsplit = 1; a.stages = 2; a.split_tiles = 1;
+    dim3 grid(H, nw, c->B);
+    ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
+    if (D == 128) {
+      static bool set_ = false;
+      if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_rows<128, ATTN_ROWS_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_rows_smem(128, ATTN_ROWS_WARPS))); set_ = true; }
+      KLAUNCH("attention_tc", (attention_rows<128, ATTN_ROWS_WARPS>), grid, dim3(ATTN_ROWS_WARPS * 32), attention_rows_smem(128, ATTN_ROWS_WARPS), a);
+    } else {
+      static bool set_ = false;
+      if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_rows<64, ATTN_ROWS_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_rows_smem(64, ATTN_ROWS_WARPS))); set_ = true; }
+      KLAUNCH("attention_tc", (attention_rows<64, ATTN_ROWS_WARPS>), grid, dim3(ATTN_ROWS_WARPS * 32), attention_rows_smem(64, ATTN_ROWS_WARPS), a);
+    }
+    return SPEC_OK;
+  }
+  // more sequences: one CTA per (sequence, head) and KV split, all query rows. Short contexts (host
+  // bound of at most attn_single_tiles tiles) get one split and no merge step; longer ones as many
+  // split CTAs as fit beside each other, of which the kernel uses min(that, tiles / split_tiles)
   const int slots1 = std::max(1, std::min(c->nsplit_attn, (SM_SLOTS / 2) / (H * c->B)));
-  a.nsplit = tiles_hi <= ATTN_SINGLE_TILES ? 1 : slots1;
+  a.nsplit = tiles_hi <= c->attn_single_tiles ? 1 : slots1;
+  a.split_tiles = c->attn_split_tiles;
   a.stages = 4;
-  a.row_blocks = 1;
-  int nw = (R + 15) / 16;
-  // short context and few sequences: a CTA per 16 query rows, its six warps taking a KV tile each,
-  // so that a head's work spreads over several SMs instead of one
-  const bool row_mode = a.nsplit == 1 && nw > 1 && nw <= 4 && H * c->B * nw <= SM_SLOTS / 2;
-  if (row_mode) { a.row_blocks = nw; a.stages = 6; }
-  dim3 grid(H, a.nsplit * a.row_blocks, c->B);
+  dim3 grid(H, a.nsplit, c->B);
 #define ATTN_CASE(HDV, NWV, KGV)                                                                         \
   {                                                                                                    \
     size_t sm = attention_tc_smem(HDV, NWV, a.stages);                                                 \
@@ -519,11 +542,9 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
     // up to 64 rows: two key groups of warps per CTA; more rows: one
     ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
     if (D == 128) {
-      if (row_mode) ATTN_CASE(128, 1, 6)
-      else if (nw <= 1) ATTN_CASE(128, 1, 2) else if (nw <= 2) ATTN_CASE(128, 2, 2) else if (nw <= 4) ATTN_CASE(128, 4, 2) else ATTN_CASE(128, 8, 1)
+      if (nw <= 1) ATTN_CASE(128, 1, 2) else if (nw <= 2) ATTN_CASE(128, 2, 2) else if (nw <= 4) ATTN_CASE(128, 4, 2) else ATTN_CASE(128, 8, 1)
     } else {
-      if (row_mode) ATTN_CASE(64, 1, 6)
-      else if (nw <= 1) ATTN_CASE(64, 1, 2) else if (nw <= 2) ATTN_CASE(64, 2, 2) else if (nw <= 4) ATTN_CASE(64, 4, 2) else ATTN_CASE(64, 8, 1)
+      if (nw <= 1) ATTN_CASE(64, 1, 2) else if (nw <= 2) ATTN_CASE(64, 2, 2) else if (nw <= 4) ATTN_CASE(64, 4, 2) else ATTN_CASE(64, 8, 1)
     }
   }
 #undef ATTN_CASE
@@ -853,7 +874,8 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   // length bounds and a recorded step serves every length below its bound
   std::vector<int> n_hi_plan(B), n_lo_plan(B);
   for (int b = 0; b < B; ++b) {
-    n_hi_plan[b] = (c->n_hi[b] + T_ <= ATTN_SINGLE_TILES * 64 ? std::min(ATTN_SINGLE_TILES * 64, c->cap) : c->cap) - T_;
+    const bool any_len = attn_rows_mode(c, T_) || c->n_hi[b] + T_ > c->attn_single_tiles * 64;
+    n_hi_plan[b] = (any_len ? c->cap : std::min(c->attn_single_tiles * 64, c->cap)) - T_;
     n_lo_plan[b] = c->n_lo[b];
   }
   const bool use_graph = c->graph_on && !c->trace_on && c->profile_kind == 0;
@@ -1115,6 +1137,8 @@ int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
   switch (what) {
     case SPEC_OPT_GRAPH:
       c->graph_on = value != 0; return SPEC_OK;
+    case 6: c->attn_split_tiles = value < 1 ? 1 : value; return SPEC_OK;
+    case 7: c->attn_single_tiles = value < 1 ? 1 : value; return SPEC_OK;
     case SPEC_OPT_PDL: c->pdl = value != 0; return SPEC_OK;
     case SPEC_OPT_GEMM_CTAS:
       if (value < 1 || value > SM_SLOTS) return c->fail(SPEC_E_BADARG, "gemm CTA count out of range");
