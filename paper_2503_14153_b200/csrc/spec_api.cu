@@ -35,6 +35,7 @@ constexpr int TRACE_CAP = 1024;     // launches of one step the timeline can hol
 constexpr int SM_SLOTS = 296;       // 148 SMs x 2 co-resident GEMM CTAs
 constexpr int MAX_STEPS_AHEAD = 8;      // enqueue-only steps the host may run ahead of the device
 constexpr int ATTN_ROWS_WARPS = 6;      // warps of the CTA-per-16-rows attention kernel
+constexpr int ATTN_SPLIT_TILES = 8;       // fewest KV tiles a split of attention_tc gets (2..8 measured alike)
 constexpr int ATTN_SINGLE_TILES = 12;   // contexts of at most this many 64-key tiles use one KV split
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -184,8 +185,6 @@ struct spec_ctx {
   bool pdl = true;                     // programmatic dependent launch between the kernels of a step
   int gemm_ctas = 288;                 // persistent CTAs of the weight-streaming GEMM (measured best; at most SM_SLOTS)
   int l2_prefetch = 0;
-  int attn_split_tiles = 8;            // fewest KV tiles a split of the attention gets
-  int attn_single_tiles = ATTN_SINGLE_TILES;
   int small_gemm_ctas = 192;           // CTAs of GEMMs with at most 48 weight tiles (Wo, down): fewer partial sums                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
   std::vector<int> h_parent, h_depth, h_rank;
   std::vector<int> n_hi, n_lo;         // host upper / lower bounds of the committed lengths
@@ -524,11 +523,11 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
     return SPEC_OK;
   }
   // more sequences: one CTA per (sequence, head) and KV split, all query rows. Short contexts (host
-  // bound of at most attn_single_tiles tiles) get one split and no merge step; longer ones as many
+  // bound of at most ATTN_SINGLE_TILES tiles) get one split and no merge step; longer ones as many
   // split CTAs as fit beside each other, of which the kernel uses min(that, tiles / split_tiles)
   const int slots1 = std::max(1, std::min(c->nsplit_attn, (SM_SLOTS / 2) / (H * c->B)));
-  a.nsplit = tiles_hi <= c->attn_single_tiles ? 1 : slots1;
-  a.split_tiles = c->attn_split_tiles;
+  a.nsplit = tiles_hi <= ATTN_SINGLE_TILES ? 1 : slots1;
+  a.split_tiles = ATTN_SPLIT_TILES;
   a.stages = 4;
   dim3 grid(H, a.nsplit, c->B);
 #define ATTN_CASE(HDV, NWV, KGV)                                                                         \
@@ -874,8 +873,8 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   // length bounds and a recorded step serves every length below its bound
   std::vector<int> n_hi_plan(B), n_lo_plan(B);
   for (int b = 0; b < B; ++b) {
-    const bool any_len = attn_rows_mode(c, T_) || c->n_hi[b] + T_ > c->attn_single_tiles * 64;
-    n_hi_plan[b] = (any_len ? c->cap : std::min(c->attn_single_tiles * 64, c->cap)) - T_;
+    const bool any_len = attn_rows_mode(c, T_) || c->n_hi[b] + T_ > ATTN_SINGLE_TILES * 64;
+    n_hi_plan[b] = (any_len ? c->cap : std::min(ATTN_SINGLE_TILES * 64, c->cap)) - T_;
     n_lo_plan[b] = c->n_lo[b];
   }
   const bool use_graph = c->graph_on && !c->trace_on && c->profile_kind == 0;
@@ -1137,8 +1136,6 @@ int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
   switch (what) {
     case SPEC_OPT_GRAPH:
       c->graph_on = value != 0; return SPEC_OK;
-    case 6: c->attn_split_tiles = value < 1 ? 1 : value; return SPEC_OK;
-    case 7: c->attn_single_tiles = value < 1 ? 1 : value; return SPEC_OK;
     case SPEC_OPT_PDL: c->pdl = value != 0; return SPEC_OK;
     case SPEC_OPT_GEMM_CTAS:
       if (value < 1 || value > SM_SLOTS) return c->fail(SPEC_E_BADARG, "gemm CTA count out of range");
