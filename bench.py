@@ -354,6 +354,36 @@ def main():
         if tr:
             out["timeline_us"]["step_span"] = round((max(r[2] for r in tr) - min(r[1] for r in tr)) / 1e3, 1)
 
+        # ---------------- context: plain autoregressive decoding on the same kernels ----------------
+        # One-node tree, no extra heads: what a token costs without speculation. The step rate of the
+        # tree-verifying decoder times the accepted length Sigma_i p^i of the controlled draft (Sec. III-B
+        # candidates accepted with probability p per head; the GPU tests check that the measured lengths
+        # follow this form) gives the tokens/s a draft of that quality would reach on this step.
+        if K > 0 and world == 1:
+            from paper_2503_14153_b200 import chain_tree
+            dec.close()
+            cfg_ar = cfg.with_(n_medusa=0, topk=(), tree_nodes=1)
+            ar = SpecDecoder(cfg_ar, dw, chain_tree(1), cfg.prompt_len + 80)
+            ar.prefill(prompt)
+            for _ in range(5):
+                ar.step_async()
+            torch.cuda.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            for _ in range(40):
+                ar.step_async()
+            a1.record(stream)
+            torch.cuda.synchronize()
+            ar_ms = a0.elapsed_time(a1) / 40
+            ar.close()
+            out["autoregressive"] = {"ms_per_step": ar_ms, "tokens_per_s": 1e3 / ar_ms,
+                                     "tree_step_over_ar_step": ms_per_step / ar_ms}
+            out["tokens_per_s_at_draft_quality"] = {
+                f"p={p}": {"accepted_len_closed_form": sum(p ** i for i in range(K + 1)),
+                           "tokens_per_s": sum(p ** i for i in range(K + 1)) * 1e3 / ms_per_step,
+                           "speedup_over_autoregressive": sum(p ** i for i in range(K + 1)) * ar_ms / ms_per_step}
+                for p in (0.3, 0.6, 0.9)}
+
     if want_cpu:
         dt, cnt, threads = oracle_step_sample(cfg, host_w, tree)
         out["cpu_baseline"] = {"value": cnt / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
