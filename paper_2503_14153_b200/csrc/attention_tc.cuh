@@ -97,9 +97,8 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
   const int ST = a.stages;
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* qs = smem;                                       // [NW*16][HD]
-  uint8_t* ks = qs + NW * 16 * ROWB;                        // [ST][KT][HD]
-  uint8_t* vs = ks + ST * TILE_BYTES;                       // [ST][KT][HD]
-  uint64_t* full = reinterpret_cast<uint64_t*>(vs + ST * TILE_BYTES);   // [ATTN_MAX_STAGES]
+  uint8_t* ks = qs + NW * 16 * ROWB;                        // [ST][page][K | V][16][HD]
+  uint64_t* full = reinterpret_cast<uint64_t*>(ks + ST * 2 * TILE_BYTES);   // [ATTN_MAX_STAGES]
   int* pt_s = reinterpret_cast<int*>(full + ATTN_MAX_STAGES);           // [ATTN_PT_CACHE] page-table entries of this split
 
   pdl_launch_dependents();
@@ -124,10 +123,9 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
     for (int pg = 0; pg < KT / 16; ++pg) {
       const int e = (tile - t0) * (KT / 16) + pg;
       const int page = e < ATTN_PT_CACHE ? pt_s[e] : pt[tile * (KT / 16) + pg];
-      bulk_load_1d(ks + buf * TILE_BYTES + pg * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 0, kvh),
-                   PAGE_BYTES, &full[buf]);
-      bulk_load_1d(vs + buf * TILE_BYTES + pg * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 1, kvh),
-                   PAGE_BYTES, &full[buf]);
+      // the K block and the V block of a (page, layer, head) are adjacent in the pool: one copy
+      bulk_load_1d(ks + buf * 2 * TILE_BYTES + pg * 2 * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 0, kvh),
+                   2 * PAGE_BYTES, &full[buf]);
     }
   };
   // tiles that lie wholly below the host's lower bound of the committed length hold rows of
@@ -217,8 +215,8 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
     if (it == 0 && threadIdx.x == 0) trace_mark_max(tr, 3);
     if (have) {
       const int t = t0 + my;
-      const uint8_t* kt = ks + (my % ST) * TILE_BYTES;
-      const uint8_t* vt = vs + (my % ST) * TILE_BYTES;
+      const uint8_t* kt = ks + (my % ST) * 2 * TILE_BYTES;   // key `key` of the tile: page key / 16, row key % 16
+      const uint8_t* vt = kt + PAGE_BYTES;
       float s[KT / 8][4];
 #pragma unroll
       for (int j = 0; j < KT / 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
@@ -231,7 +229,7 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
           for (int j2 = 0; j2 < KT / 16; ++j2) {
             int key = j2 * 16 + (lane & 7) + (lane >> 4) * 8;
             int ch = kk * 2 + ((lane >> 3) & 1);
-            ldmatrix_x4(smem_u32(kt + key * ROWB + ((ch ^ (key & 7)) << 4)), dst[j2]);
+            ldmatrix_x4(smem_u32(kt + (key >> 4) * 2 * PAGE_BYTES + (key & 15) * ROWB + ((ch ^ (key & 7)) << 4)), dst[j2]);
           }
         };
         load_k(0, kf[0]);
@@ -296,7 +294,7 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
           for (int dd = 0; dd < DG; ++dd) {
             int key = j * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
             int ch = (d0 + dd) * 2 + (lane >> 4);
-            ldmatrix_x4_trans(smem_u32(vt + key * ROWB + ((ch ^ (key & 7)) << 4)), dst[dd]);
+            ldmatrix_x4_trans(smem_u32(vt + (key >> 4) * 2 * PAGE_BYTES + (key & 15) * ROWB + ((ch ^ (key & 7)) << 4)), dst[dd]);
           }
         };
         load_v(0, vf[0]);
@@ -485,7 +483,7 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
   constexpr int NTHR = W * 32;
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* qs = smem;                                                        // [16][HD]
-  uint8_t* kv = qs + 16 * ROWB;                                              // [W][NB][K | V][SK][HD]
+  uint8_t* kv = qs + 16 * ROWB;                                              // [W][NB][page][K | V][16][HD]
   uint64_t* full = reinterpret_cast<uint64_t*>(kv + W * NB * 2 * SUB_BYTES); // [W][NB]
   int* pt_s = reinterpret_cast<int*>(full + W * NB);                         // [ATTN_PT_CACHE]
 
@@ -508,8 +506,8 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
     for (int pg = 0; pg < SK / 16; ++pg) {
       const int e = st * (SK / 16) + pg;
       const int page = e < ATTN_PT_CACHE ? pt_s[e] : pt[e];
-      bulk_load_1d(mine + bf * 2 * SUB_BYTES + pg * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 0, kvh), PAGE_BYTES, &my_full[bf]);
-      bulk_load_1d(mine + bf * 2 * SUB_BYTES + SUB_BYTES + pg * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 1, kvh), PAGE_BYTES, &my_full[bf]);
+      // the K block and the V block of a (page, layer, head) are adjacent in the pool: one copy
+      bulk_load_1d(mine + bf * 2 * SUB_BYTES + pg * 2 * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 0, kvh), 2 * PAGE_BYTES, &my_full[bf]);
     }
   };
   // own sub-tiles that lie wholly below the host's lower bound hold rows of earlier steps
@@ -579,8 +577,8 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
     const int bf = k % NB;
     if (!mbar_wait(&my_full[bf], (k / NB) & 1, a.status, 20)) { ok = false; break; }
     if (st == 0 && lane == 0) trace_mark_max(tr, 3);
-    const uint8_t* kt = mine + bf * 2 * SUB_BYTES;
-    const uint8_t* vt = kt + SUB_BYTES;
+    const uint8_t* kt = mine + bf * 2 * SUB_BYTES;     // key `key` of the sub-tile: page key / 16, row key % 16
+    const uint8_t* vt = kt + PAGE_BYTES;
     float s[SK / 8][4];
 #pragma unroll
     for (int j = 0; j < SK / 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
@@ -592,7 +590,7 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
         for (int j2 = 0; j2 < SK / 16; ++j2) {
           const int key = j2 * 16 + (lane & 7) + (lane >> 4) * 8;
           const int ch = kk * 2 + ((lane >> 3) & 1);
-          ldmatrix_x4(smem_u32(kt + key * ROWB + ((ch ^ (key & 7)) << 4)), dst[j2]);
+          ldmatrix_x4(smem_u32(kt + (key >> 4) * 2 * PAGE_BYTES + (key & 15) * ROWB + ((ch ^ (key & 7)) << 4)), dst[j2]);
         }
       };
       load_k(0, kf[0]);
@@ -656,7 +654,7 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
         for (int dd = 0; dd < DG; ++dd) {
           const int key = j * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
           const int ch = (d0 + dd) * 2 + (lane >> 4);
-          ldmatrix_x4_trans(smem_u32(vt + key * ROWB + ((ch ^ (key & 7)) << 4)), dst[dd]);
+          ldmatrix_x4_trans(smem_u32(vt + (key >> 4) * 2 * PAGE_BYTES + (key & 15) * ROWB + ((ch ^ (key & 7)) << 4)), dst[dd]);
         }
       };
       load_v(0, vf[0]);
