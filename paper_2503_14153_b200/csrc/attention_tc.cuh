@@ -606,18 +606,30 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
     }
     // mask + online softmax (log2 domain)
     const int k0 = st * SK;
-    uint32_t vis0 = ~0u, vis1 = ~0u;
-    if (k0 + SK > n) { vis0 = (uint32_t)attn_vis64(anc0, k0, n); vis1 = (uint32_t)attn_vis64(anc1, k0, n); }
     float tmax[2] = {-INFINITY, -INFINITY};
+    if (k0 + SK > n) {
+      // the sub-tile reaches into the tree rows: per-key visibility
+      const uint32_t vis0 = (uint32_t)attn_vis64(anc0, k0, n), vis1 = (uint32_t)attn_vis64(anc1, k0, n);
 #pragma unroll
-    for (int j = 0; j < SK / 8; ++j) {
+      for (int j = 0; j < SK / 8; ++j) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float v = s[j][e] * a.scale_log2;
-        const int bi = j * 8 + (lane & 3) * 2 + (e & 1);
-        if (!(((e < 2 ? vis0 : vis1) >> bi) & 1u)) v = -INFINITY;
-        s[j][e] = v;
-        tmax[e >> 1] = fmaxf(tmax[e >> 1], v);
+        for (int e = 0; e < 4; ++e) {
+          float v = s[j][e] * a.scale_log2;
+          const int bi = j * 8 + (lane & 3) * 2 + (e & 1);
+          if (!(((e < 2 ? vis0 : vis1) >> bi) & 1u)) v = -INFINITY;
+          s[j][e] = v;
+          tmax[e >> 1] = fmaxf(tmax[e >> 1], v);
+        }
+      }
+    } else {
+      // committed positions only: every key is visible to every row
+#pragma unroll
+      for (int j = 0; j < SK / 8; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          s[j][e] *= a.scale_log2;
+          tmax[e >> 1] = fmaxf(tmax[e >> 1], s[j][e]);
+        }
       }
     }
     float alpha[2], mnew[2];
