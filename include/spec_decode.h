@@ -63,6 +63,10 @@ typedef struct {
 
 #define SPEC_FLAG_KEEP_LOGITS 1 /* materialise verify logits [rows, vocab] for spec_debug_read  */
 #define SPEC_FLAG_SIMPLE_KERNELS 2 /* bf16: run the plain CUDA-core kernels (debug aid, slow)  */
+#define SPEC_FLAG_PACKED_WEIGHTS 4 /* bf16 tensor-core path: every linear weight pointer of spec_weights
+                                      (wq, wk, wv, wo, w_gate, w_up, w_down, lm_head, medusa_w) is the
+                                      pre-tiled image made by spec_pack_weight, not the row-major matrix
+                                      (embed, norms and biases stay as they are)                    */
 
 /* Candidate tree, HOST arrays of n_nodes entries, copied at spec_create. Rules: node 0 is
  * the root (parent -1, depth 0, rank 0) and carries the base model's own next token;
@@ -208,6 +212,20 @@ int spec_debug_read_kv(spec_ctx *ctx, int32_t seq, int32_t layer, int32_t slot0,
                        float *host_k, float *host_v);
 
 /* ---- single operations of the verify forward, for unit parity tests and profiling ---- */
+
+/* Pre-tiled weights. The paper has no counterpart: it is a storage layout for this library's GEMM.
+ * The weight stream of a step reads every matrix once, tile by tile; out of a row-major matrix
+ * a tile is 128 separate 128-byte pieces, which the memory system serves at about 6.4 TB/s. In the
+ * pre-tiled image each (128-row tile, 64-column K chunk) unit is 16 KiB contiguous, already in the
+ * shared-memory layout the tensor cores read, and a CTA's run of units is one contiguous stretch:
+ * about 7.3 TB/s. spec_packed_weight_bytes: size of the image of a [rows, cols] bf16 matrix
+ * (cols % 64 == 0; rows are padded to a multiple of 128 with zeros), 0 if the shape is not
+ * supported. spec_pack_weight: w DEVICE bf16 row-major [rows, cols] -> packed DEVICE (16-byte
+ * aligned, spec_packed_weight_bytes bytes, must not overlap w), enqueued on `cuda_stream`. The
+ * caller owns both buffers and may free w afterwards. A context created with
+ * SPEC_FLAG_PACKED_WEIGHTS takes images instead of matrices. */
+size_t spec_packed_weight_bytes(int32_t rows, int32_t cols);
+int spec_pack_weight(const void *w, int32_t rows, int32_t cols, void *packed, void *cuda_stream);
 
 /* y[M,N] (float32, DEVICE) = x[M,K] * W[N,K]^T for DEVICE x and W of type `dtype`
  * (Sec. III-B verification forward: every projection of the base model). bf16 runs the

@@ -7,4 +7,5 @@ loudly if it has not been built.
 """
 from .tree import build_tree, chain_tree  # noqa: F401
 from .binding import (SpecDecoder, SpecError, load_library, library_path, spec_op_linear, spec_op_linear_static, spec_build_labels,  # noqa: F401
-                      upload_weights, FLAG_KEEP_LOGITS, FLAG_SIMPLE_KERNELS)
+                      upload_weights, FLAG_KEEP_LOGITS, FLAG_SIMPLE_KERNELS, FLAG_PACKED_WEIGHTS,
+                      spec_pack_weight, pack_linear_weights)

@@ -16,6 +16,7 @@ _lib = None
 
 FLAG_KEEP_LOGITS = 1
 FLAG_SIMPLE_KERNELS = 2
+FLAG_PACKED_WEIGHTS = 4
 PROFILE_OFF, PROFILE_GATE_UP, PROFILE_QKV, PROFILE_WO, PROFILE_DOWN, PROFILE_ATTENTION = range(6)
 
 Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB, Q_GRAPH_CAPTURES = 0, 1, 2, 3, 4, 5
@@ -26,7 +27,8 @@ TRACE_NAME_LEN = 32
 
 EXPORTS = ["spec_workspace_bytes", "spec_create", "spec_prefill", "spec_step", "spec_read_generated",
            "spec_destroy", "spec_last_error", "spec_query", "spec_debug_read", "spec_debug_read_kv",
-           "spec_op_linear", "spec_op_linear_scratch_floats", "spec_op_linear_static", "spec_set_option", "spec_trace_read", "spec_build_labels", "spec_last_step_phase_ms", "spec_profile_kernel",
+           "spec_op_linear", "spec_op_linear_scratch_floats", "spec_op_linear_static", "spec_packed_weight_bytes",
+           "spec_pack_weight", "spec_set_option", "spec_trace_read", "spec_build_labels", "spec_last_step_phase_ms", "spec_profile_kernel",
            "spec_profile_read"]
 
 
@@ -105,6 +107,10 @@ def load_library():
     lib.spec_op_linear_static.restype = C.c_int
     lib.spec_op_linear_static.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_void_p]
+    lib.spec_packed_weight_bytes.restype = C.c_size_t
+    lib.spec_packed_weight_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.spec_pack_weight.restype = C.c_int
+    lib.spec_pack_weight.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     lib.spec_last_step_phase_ms.restype = C.c_int
     lib.spec_last_step_phase_ms.argtypes = [C.c_void_p, C.c_void_p]
     lib.spec_profile_kernel.restype = C.c_int
@@ -146,13 +152,61 @@ def upload_weights(cfg, weights: Dict[str, np.ndarray], device="cuda:0") -> Dict
     return out
 
 
+def spec_pack_weight(w):
+    """Pre-tiled image (uint8 CUDA tensor) of a row-major bf16 CUDA matrix, made by the library."""
+    import torch
+    lib = load_library()
+    rows, cols = w.shape
+    nbytes = int(lib.spec_packed_weight_bytes(rows, cols))
+    if nbytes == 0 or w.dtype != torch.bfloat16 or not w.is_contiguous():
+        raise SpecError(-1, "spec_pack_weight: needs a contiguous bf16 matrix whose width is a multiple of 64")
+    out = torch.empty(nbytes, dtype=torch.uint8, device=w.device)
+    rc = lib.spec_pack_weight(w.data_ptr(), rows, cols, out.data_ptr(), torch.cuda.current_stream(w.device).cuda_stream)
+    if rc != 0:
+        raise SpecError(rc, lib.spec_last_error(None).decode())
+    return out
+
+
+def pack_linear_weights(cfg, dev_weights: Dict[str, "object"]) -> Dict[str, "object"]:
+    """Pre-tiled images of every linear weight of the model (q, k and v separately), keyed like the
+    pointers of spec_weights; cached on the weight dictionary, so decoders that share weights share
+    the images."""
+    cache = dev_weights.get("__packed__")
+    if cache is not None:
+        return cache
+    qrows, krows = cfg.n_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim
+    out = {"lm_head": spec_pack_weight(dev_weights["lm_head"])}
+    for l in range(cfg.n_layers):
+        p = f"layers.{l}."
+        qkv = dev_weights[p + "wqkv"]
+        out[p + "wq"] = spec_pack_weight(qkv[:qrows])
+        out[p + "wk"] = spec_pack_weight(qkv[qrows:qrows + krows])
+        out[p + "wv"] = spec_pack_weight(qkv[qrows + krows:])
+        for nm in ("wo", "w_gate", "w_up", "w_down"):
+            out[p + nm] = spec_pack_weight(dev_weights[p + nm])
+    for k in range(cfg.n_medusa):
+        out[f"medusa.{k}.w"] = spec_pack_weight(dev_weights[f"medusa.{k}.w"])
+    import torch
+    torch.cuda.synchronize()      # whatever stream a decoder runs on, the images are complete
+    dev_weights["__packed__"] = out
+    return out
+
+
 class SpecDecoder:
-    """Owns the device tensors and a spec_ctx; methods mirror the C entry points."""
+    """Owns the device tensors and a spec_ctx; methods mirror the C entry points. On the bf16 tensor-core
+    path the linear weights are handed over as pre-tiled images unless packed=False."""
 
     def __init__(self, cfg, dev_weights: Dict[str, "object"], tree: Dict[str, np.ndarray], max_seq: int,
                  max_batch: int = 1, flags: int = 0, accept_mode: int = 0, typ_eps: float = 0.09,
-                 typ_delta: float = 0.3, temperature: float = 1.0, frag_token: int = -1, stream=None):
+                 typ_delta: float = 0.3, temperature: float = 1.0, frag_token: int = -1, stream=None,
+                 packed: Optional[bool] = None):
         import torch
+        tc_path = cfg.dtype == "bf16" and not (flags & FLAG_SIMPLE_KERNELS)
+        self.packed = tc_path if packed is None else bool(packed)
+        if self.packed:
+            if not tc_path:
+                raise SpecError(-1, "pre-tiled weights need the bf16 tensor-core path")
+            flags |= FLAG_PACKED_WEIGHTS
         self.torch = torch
         self.lib = load_library()
         self.cfg = cfg
@@ -178,17 +232,27 @@ class SpecDecoder:
             return a
 
         lw = lambda nm: [dev_weights[f"layers.{l}.{nm}"].data_ptr() for l in range(L)]
-        qkv = lw("wqkv")
+        if self.packed:
+            self._pk = pack_linear_weights(cfg, dev_weights)
+            pw = lambda nm: [self._pk[f"layers.{l}.{nm}"].data_ptr() for l in range(L)]
+            lin = {nm: pw(nm) for nm in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")}
+            medusa_w = [self._pk[f"medusa.{k}.w"].data_ptr() for k in range(self.K)]
+            lm_head_ptr = self._pk["lm_head"].data_ptr()
+        else:
+            qkv = lw("wqkv")
+            lin = {"wq": qkv, "wk": [p + qrows * cfg.d_model * esz for p in qkv],
+                   "wv": [p + (qrows + krows) * cfg.d_model * esz for p in qkv],
+                   "wo": lw("wo"), "w_gate": lw("w_gate"), "w_up": lw("w_up"), "w_down": lw("w_down")}
+            medusa_w = [dev_weights[f"medusa.{k}.w"].data_ptr() for k in range(self.K)]
+            lm_head_ptr = dev_weights["lm_head"].data_ptr()
         self._arrs = {
-            "attn_norm": arr(lw("attn_norm")), "wq": arr(qkv),
-            "wk": arr([p + qrows * cfg.d_model * esz for p in qkv]),
-            "wv": arr([p + (qrows + krows) * cfg.d_model * esz for p in qkv]),
-            "wo": arr(lw("wo")), "ffn_norm": arr(lw("ffn_norm")), "w_gate": arr(lw("w_gate")),
-            "w_up": arr(lw("w_up")), "w_down": arr(lw("w_down")),
-            "medusa_w": arr([dev_weights[f"medusa.{k}.w"].data_ptr() for k in range(self.K)]),
+            "attn_norm": arr(lw("attn_norm")), "wq": arr(lin["wq"]), "wk": arr(lin["wk"]), "wv": arr(lin["wv"]),
+            "wo": arr(lin["wo"]), "ffn_norm": arr(lw("ffn_norm")), "w_gate": arr(lin["w_gate"]),
+            "w_up": arr(lin["w_up"]), "w_down": arr(lin["w_down"]),
+            "medusa_w": arr(medusa_w),
             "medusa_b": arr([dev_weights[f"medusa.{k}.b"].data_ptr() for k in range(self.K)]),
         }
-        self._cw = SpecWeights(dev_weights["embed"].data_ptr(), dev_weights["lm_head"].data_ptr(),
+        self._cw = SpecWeights(dev_weights["embed"].data_ptr(), lm_head_ptr,
                                dev_weights["final_norm"].data_ptr(),
                                *[C.cast(self._arrs[n], C.POINTER(C.c_void_p)) for n in
                                  ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down",

@@ -46,6 +46,11 @@ struct StreamGemmParams {
   int mat_col0[GS_MAX_MATS];        // first logical output column of each matrix
   int n_tiles;
   SegMap seg;
+  // Pre-tiled weights (see pack_weight_tiles): packed[i] != nullptr holds matrix i as the sequence of its
+  // (tile, K chunk) units, each the 16 KB shared-memory image of the tile (128 rows of 128 bytes, 16-byte
+  // chunks XOR-swizzled with the row). A CTA's run of units is then one contiguous stretch of memory read
+  // with plain bulk copies, which streams faster out of HBM than strided TMA boxes (7.3 against 6.4 TB/s).
+  const uint8_t* packed[GS_MAX_MATS];
   int l2_prefetch;                  // units to request into L2 beyond the ring before the dependency wait
   // partial sums: part[slot][m][n_tiles*128] (padded column space: tile nt owns columns [128 nt, 128 nt + 128))
   float* part;
@@ -121,7 +126,7 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
     mbar_init(&acc_full[0], 1); mbar_init(&acc_full[1], 1);
     mbar_init(&acc_empty[0], 4); mbar_init(&acc_empty[1], 4);
     mbar_fence_init();
-    for (int i = 0; i < p.n_mats; ++i) tma_prefetch_desc(&tm.a[i]);
+    for (int i = 0; i < p.n_mats; ++i) if (!p.packed[i]) tma_prefetch_desc(&tm.a[i]);
     tma_prefetch_desc(&tm.b);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, Cfg::TMEM_COLS); tmem_relinquish(); }
@@ -136,18 +141,24 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
       const int n_units = hi - lo;
       const uint64_t wpol = l2_policy_evict_first();
       const int n_pre = n_units < STAGES ? n_units : STAGES;
+      auto load_a = [&](uint8_t* dst, const GsUnit& w, uint64_t* bar) {
+        if (p.packed[w.mat])
+          bulk_load_1d_hint(dst, p.packed[w.mat] + ((size_t)(w.row0 >> 7) * KC + w.kc) * Cfg::A_BYTES, Cfg::A_BYTES, bar, wpol);
+        else
+          tma_load_2d_hint(dst, &tm.a[w.mat], w.kc * Cfg::BK, w.row0, bar, wpol);
+      };
       // weights first: they do not depend on the kernel before this one
       for (int i = 0; i < n_pre; ++i) {
         GsUnit w = gs_decode(p, lo + i);
         mbar_expect_tx(&full[i], Cfg::STAGE_BYTES);
-        tma_load_2d_hint(tiles + i * Cfg::STAGE_BYTES, &tm.a[w.mat], w.kc * Cfg::BK, w.row0, &full[i], wpol);
+        load_a(tiles + i * Cfg::STAGE_BYTES, w, &full[i]);
       }
       {
         int n_pf = n_units - n_pre;
         if (n_pf > p.l2_prefetch) n_pf = p.l2_prefetch;
         for (int i = 0; i < n_pf; ++i) {
           GsUnit w = gs_decode(p, lo + n_pre + i);
-          tma_prefetch_l2_2d(&tm.a[w.mat], w.kc * Cfg::BK, w.row0, wpol);
+          if (!p.packed[w.mat]) tma_prefetch_l2_2d(&tm.a[w.mat], w.kc * Cfg::BK, w.row0, wpol);
         }
       }
       pdl_wait();
@@ -164,7 +175,7 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
         GsUnit w = gs_decode(p, lo + issued);
         uint8_t* a = tiles + st * Cfg::STAGE_BYTES;
         mbar_expect_tx(&full[st], Cfg::STAGE_BYTES);
-        tma_load_2d_hint(a, &tm.a[w.mat], w.kc * Cfg::BK, w.row0, &full[st], wpol);
+        load_a(a, w, &full[st]);
         tma_load_2d(a + Cfg::A_BYTES, &tm.b, w.kc * Cfg::BK, w.mt * MT, &full[st]);
       }
       if (!ok) {
@@ -259,6 +270,24 @@ gemm_stream(const __grid_constant__ StreamTmaps tm, const StreamGemmParams p) {
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+}
+
+// Writes the pre-tiled image of a row-major bf16 matrix [rows][cols] (cols % 64 == 0): unit (tile t, K chunk
+// kc) at byte offset (t * cols / 64 + kc) * 16384, row r of the tile at r * 128, its 16-byte chunk c at chunk
+// position c ^ (r & 7) -- what a TMA load with the 128-byte swizzle leaves in shared memory. Rows beyond the
+// matrix are zeros. One CTA per unit.
+__global__ void __launch_bounds__(256)
+pack_weight_tiles(const bf16* __restrict__ w, int rows, int cols, uint8_t* __restrict__ packed) {
+  const int KC = cols >> 6;
+  const int t = blockIdx.x / KC, kc = blockIdx.x - t * KC;
+  uint4* dst = reinterpret_cast<uint4*>(packed + (size_t)blockIdx.x * 16384);
+  for (int i = threadIdx.x; i < 128 * 8; i += blockDim.x) {
+    const int r = i >> 3, ch = i & 7;
+    const int row = t * 128 + r;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (row < rows) v = *reinterpret_cast<const uint4*>(w + (size_t)row * cols + kc * 64 + ch * 8);
+    dst[r * 8 + (ch ^ (r & 7))] = v;
+  }
 }
 
 }  // namespace spec

@@ -182,6 +182,7 @@ struct spec_ctx {
   size_t esz;                          // operand element size
   int Mcap, cap, pages_per_seq, gen_cap, nsplit_attn, Nqkv, ntile_lm, topk_slice, topk_blocks;
   bool qkv_fused, keep_logits;
+  bool packed = false;                 // linear weights are pre-tiled images (SPEC_FLAG_PACKED_WEIGHTS)
   bool pdl = true;                     // programmatic dependent launch between the kernels of a step
   int gemm_ctas = 288;                 // persistent CTAs of the weight-streaming GEMM (measured best; at most SM_SLOTS)
   int l2_prefetch = 0;
@@ -293,6 +294,7 @@ bool validate_config(const spec_config* c, std::string* why) {
   if (c->n_medusa < 0 || c->n_medusa > SPEC_MAX_HEADS) { *why = "n_medusa out of range"; return false; }
   if (c->accept_mode != 0 && c->accept_mode != 1) { *why = "accept_mode must be 0 or 1"; return false; }
   bool tc = c->dtype == 1 && !(c->flags & SPEC_FLAG_SIMPLE_KERNELS);
+  if ((c->flags & SPEC_FLAG_PACKED_WEIGHTS) && !tc) { *why = "pre-tiled weights need the bf16 tensor-core path"; return false; }
   if (tc) {
     if (c->d_model % 64 || c->d_ffn % 64 || (c->n_heads * c->head_dim) % 64) { *why = "bf16 path needs widths that are multiples of 64"; return false; }
     if (c->head_dim != 64 && c->head_dim != 128) { *why = "bf16 path needs head_dim 64 or 128"; return false; }
@@ -444,6 +446,7 @@ int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* c
   if (plan_part_floats(g) > c->part_floats) return c->fail(SPEC_E_NOMEM, "partial-sum scratch too small");
   StreamTmaps tm{};
   for (int i = 0; i < n_mats; ++i) {
+    if (c->packed) { g.p.packed[i] = static_cast<const uint8_t*>(mats[i]); continue; }
     const CUtensorMap* t = c->tmap(mats[i], rows[i], K, 128);
     if (!t) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed (weights)");
     tm.a[i] = *t;
@@ -991,6 +994,7 @@ int spec_create(const spec_config* cfg, const spec_weights* w, const spec_tree* 
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->T = tree->n_nodes; c->K = cfg->n_medusa; c->kmax = kmax; c->B = cfg->max_batch;
   c->tc = cfg->dtype == 1 && !(cfg->flags & SPEC_FLAG_SIMPLE_KERNELS);
+  c->packed = (cfg->flags & SPEC_FLAG_PACKED_WEIGHTS) != 0;
   c->esz = cfg->dtype == 1 ? 2 : 4;
   size_t need = carve(c, workspace);
   if (need > workspace_bytes) { g_create_error = "workspace too small"; delete c; return SPEC_E_NOMEM; }
@@ -1301,6 +1305,26 @@ int spec_build_labels(const int32_t* tokens, int32_t n_seq, int32_t seq_len, int
   build_labels_kernel<<<grid, LABEL_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(tokens, seq_len, num_heads, frag_token,
                                                                                         pad_token, ignore_token, labels);
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_E_CUDA;
+}
+
+size_t spec_packed_weight_bytes(int32_t rows, int32_t cols) {
+  if (rows < 1 || cols < 64 || cols % 64) return 0;
+  return (size_t)((rows + 127) / 128) * (size_t)(cols / 64) * 16384;
+}
+
+int spec_pack_weight(const void* w, int32_t rows, int32_t cols, void* packed, void* cuda_stream) {
+  const size_t bytes = spec_packed_weight_bytes(rows, cols);
+  if (!w || !packed || bytes == 0 || (reinterpret_cast<uintptr_t>(packed) & 15) || (reinterpret_cast<uintptr_t>(w) & 15)) {
+    g_create_error = "spec_pack_weight: null or unaligned pointer, or cols not a multiple of 64";
+    return SPEC_E_BADARG;
+  }
+  const size_t units = bytes / 16384;
+  if (units > 0x7fffffffu) { g_create_error = "spec_pack_weight: matrix too large"; return SPEC_E_BADARG; }
+  pack_weight_tiles<<<(unsigned)units, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(static_cast<const bf16*>(w), rows, cols,
+                                                                                        static_cast<uint8_t*>(packed));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { g_create_error = std::string("pack_weight_tiles: ") + cudaGetErrorString(e); return SPEC_E_CUDA; }
+  return SPEC_OK;
 }
 
 size_t spec_op_linear_scratch_floats(int32_t M, int32_t N, int32_t K, int32_t ctas) {

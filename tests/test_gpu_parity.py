@@ -301,3 +301,43 @@ def test_step_graph_replay(torch):
     d1.step()
     assert d1.query(B.Q_GRAPH_CAPTURES) == 4
     d1.close()
+
+
+def test_packed_weight_image_and_equivalence(torch):
+    """spec_pack_weight writes, unit by unit, the shared-memory image a swizzled TMA load of the tile
+    leaves (checked against a NumPy construction of that layout, ragged last tile zero-filled); a
+    decoder on pre-tiled weights emits bit-identical results to one on the row-major matrices."""
+    from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights, spec_pack_weight
+    from paper_2503_14153_b200 import binding as B
+    rows, cols = 300, 192
+    rng = np.random.default_rng(5)
+    w = torch.from_numpy(rng.standard_normal((rows, cols)).astype(np.float32)).cuda().bfloat16().contiguous()
+    img = spec_pack_weight(w).cpu().numpy().view(np.uint16)
+    src = w.view(torch.int16).cpu().numpy().view(np.uint16)
+    tiles, KC = (rows + 127) // 128, cols // 64
+    want = np.zeros((tiles, KC, 128, 8, 8), dtype=np.uint16)          # [tile][kc][row][chunk position][8 elements]
+    for t in range(tiles):
+        for kc in range(KC):
+            for r in range(128):
+                if t * 128 + r < rows:
+                    for ch in range(8):
+                        want[t, kc, r, ch ^ (r & 7)] = src[t * 128 + r, kc * 64 + ch * 8: kc * 64 + ch * 8 + 8]
+    assert img.size == want.size and np.array_equal(img, want.reshape(-1))
+
+    cfg = SMALL_BF16_D128
+    dw = upload_weights(cfg, draw_weights(cfg))
+    tree = build_tree(cfg.topk, cfg.tree_nodes)
+    prompt = draw_prompt(cfg, 90)
+    outs = []
+    for packed in (True, False):
+        dec = SpecDecoder(cfg, dw, tree, 300, flags=B.FLAG_KEEP_LOGITS, packed=packed)
+        assert dec.packed == packed
+        dec.prefill(prompt)
+        toks = []
+        for _ in range(5):
+            tok, cnt = dec.step()
+            toks.extend(int(x) for x in tok[0][: int(cnt[0])])
+        outs.append((toks, dec.debug(B.DBG_LOGITS).copy(), dec.debug(B.DBG_HIDDEN).copy()))
+        dec.close()
+    assert outs[0][0] == outs[1][0]
+    assert np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][2], outs[1][2])
