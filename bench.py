@@ -276,6 +276,7 @@ def main():
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "layers": cfg.n_layers, "d_model": cfg.d_model, "tree_nodes": T,
                    "medusa_heads": K, "prompt_len": cfg.prompt_len, "batch": 1, "page_size": cfg.page_size,
+                   "weight_layout": "pre-tiled (spec_pack_weight)" if dec.packed else "row-major",
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": "weights streamed per step (13.6 GB) exceed the 126 MB L2; no flush needed"},
         "gpu_launches": int(launches),
@@ -317,12 +318,12 @@ def main():
         dec.profile_kernel(B.PROFILE_OFF)
         if k_n > 0:
             per = k_ms / k_n * 1e-3
-            out["roofline"] = {"bound": "hbm", "kernel": "gemm_stream<64> on the gate+up projection (2 x [11008,4096] bf16 weights streamed once)",
+            out["roofline"] = {"bound": "hbm", "kernel": "gemm_stream<64> on the gate+up projection (2 x [11008,4096] bf16 weights, pre-tiled, streamed once)",
                                "achieved": gate_up_b / per / 1e9, "peak": peak, "unit": "GB/s",
                                "frac": gate_up_b / per / 1e9 / peak,
                                # dram__bytes_read.sum + dram__bytes_write.sum of this kernel at this shape
                                # (profiles/gemm_stream_7b_shapes_ncu_full.md); null for other shapes
-                               "traffic": 189.9e6 if (cfg.d_model, cfg.d_ffn, T) == (4096, 11008, 64) else None,
+                               "traffic": 188.0e6 if (cfg.d_model, cfg.d_ffn, T) == (4096, 11008, 64) else None,
                                "peak_kind": peak_kind,
                                "launches_timed": int(k_n), "us_per_launch": per * 1e6,
                                "algorithmic_bytes_per_launch": gate_up_b}
