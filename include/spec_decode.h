@@ -151,7 +151,7 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
 /* Tuning knobs of a context (defaults in brackets). SPEC_OPT_PDL [1]: launch the kernels of
  * a step with programmatic dependent launch, so that each kernel's set-up and weight prefetch
  * overlap the tail of the one before. SPEC_OPT_GEMM_CTAS [288]: persistent CTAs the
- * weight-streaming GEMM deals its work to (1..296); SPEC_OPT_SMALL_GEMM_CTAS [192]: the same for
+ * weight-streaming GEMM deals its work to (1..296); SPEC_OPT_SMALL_GEMM_CTAS [288]: the same for
  * GEMMs of at most 48 weight tiles (the output and down projections), where fewer CTAs mean
  * fewer partial sums to add. SPEC_OPT_L2_PREFETCH [0]: 16 KiB weight
  * chunks each GEMM CTA requests into L2, beyond its shared-memory ring, before it waits for the

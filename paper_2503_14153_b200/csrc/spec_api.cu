@@ -186,7 +186,7 @@ struct spec_ctx {
   bool pdl = true;                     // programmatic dependent launch between the kernels of a step
   int gemm_ctas = 288;                 // persistent CTAs of the weight-streaming GEMM (measured best; at most SM_SLOTS)
   int l2_prefetch = 0;
-  int small_gemm_ctas = 192;           // CTAs of GEMMs with at most 48 weight tiles (Wo, down): fewer partial sums                 // weight chunks a GEMM CTA asks into L2 before its dependency wait
+  int small_gemm_ctas = 288;           // CTAs of GEMMs with at most 48 weight tiles (Wo, down); 288 since the weights are pre-tiled (192 before)
   std::vector<int> h_parent, h_depth, h_rank;
   std::vector<int> n_hi, n_lo;         // host upper / lower bounds of the committed lengths
   std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, mw, mb;
