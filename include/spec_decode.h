@@ -150,10 +150,11 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
 
 /* Tuning knobs of a context (defaults in brackets). SPEC_OPT_PDL [1]: launch the kernels of
  * a step with programmatic dependent launch, so that each kernel's set-up and weight prefetch
- * overlap the tail of the one before. SPEC_OPT_GEMM_CTAS [288]: persistent CTAs the
- * weight-streaming GEMM deals its work to (1..296); SPEC_OPT_SMALL_GEMM_CTAS [288]: the same for
- * GEMMs of at most 48 weight tiles (the output and down projections), where fewer CTAs mean
- * fewer partial sums to add. SPEC_OPT_L2_PREFETCH [0]: 16 KiB weight
+ * overlap the tail of the one before. SPEC_OPT_GEMM_CTAS [288]: upper bound of the persistent
+ * CTAs the weight-streaming GEMM deals its work to (1..296; the library takes the largest count
+ * within 15% of it whose runs end on tile boundaries, e.g. 258 = 3 CTAs per 2 tiles for the 172
+ * gate+up tiles); SPEC_OPT_SMALL_GEMM_CTAS [288]: the same for GEMMs of at most 48 weight tiles
+ * (the output and down projections). SPEC_OPT_L2_PREFETCH [0]: 16 KiB weight
  * chunks each GEMM CTA requests into L2, beyond its shared-memory ring, before it waits for the
  * previous kernel (0..64). Results do not depend on SPEC_OPT_PDL or SPEC_OPT_L2_PREFETCH;
  * SPEC_OPT_GEMM_CTAS and SPEC_OPT_SMALL_GEMM_CTAS change the order in which partial sums are added. SPEC_OPT_TRACE [0]:

@@ -434,6 +434,20 @@ const char* gemm_kind_name(int kind) {
   }
 }
 
+// CTA count for a GEMM of n_tiles weight tiles, at most cap: one that lets the CTAs' runs end on tile
+// boundaries (p CTAs per q tiles, q as small as possible), so that a tile's partial sums come from as few
+// CTAs as possible and the consumers read fewer slots; within 15% of cap, else cap itself.
+int aligned_ctas(int n_tiles, int cap) {
+  for (int q = 1; q <= 4; ++q) {
+    long long p = (long long)cap * q / n_tiles;
+    while (p >= 1 && (n_tiles * p) % q) --p;
+    if (p < 1) continue;
+    const int G = (int)(n_tiles * p / q);
+    if (G * 100 >= cap * 85) return G;
+  }
+  return cap;
+}
+
 // ---- tensor-core linear (bf16): partial sums of x[M,K] * [mats]^T ----
 // kind: SPEC_PROFILE_* of the call site. On success *view describes the partial sums.
 int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* const* mats, const int* rows, int kind,
@@ -441,7 +455,8 @@ int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* c
   GemmPlan g;
   int tiles_all = 0;
   for (int i = 0; i < n_mats; ++i) tiles_all += (rows[i] + 127) / 128;
-  if (!plan_gemm(M, K, n_mats, rows, tiles_all <= 48 ? std::min(c->gemm_ctas, c->small_gemm_ctas) : c->gemm_ctas, &g))
+  const int g_cap = aligned_ctas(tiles_all, tiles_all <= 48 ? std::min(c->gemm_ctas, c->small_gemm_ctas) : c->gemm_ctas);
+  if (!plan_gemm(M, K, n_mats, rows, g_cap, &g))
     return c->fail(SPEC_E_BADARG, "unsupported linear shape");
   if (plan_part_floats(g) > c->part_floats) return c->fail(SPEC_E_NOMEM, "partial-sum scratch too small");
   StreamTmaps tm{};
