@@ -162,9 +162,11 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
  * kernel sequence of a step into a CUDA graph once and replay it on the following steps (a new
  * recording when a sequence grows past the 768 positions the single-split attention launch covers,
  * after a prefill and after an option change; steps that are traced or profiled are enqueued
- * directly). Results do not depend on it. */
+ * directly). Results do not depend on it. SPEC_OPT_PHASE_TIMING [0]: record an event at the five
+ * phase boundaries of every step for spec_last_step_phase_ms (costs the programmatic overlap at
+ * those boundaries: about 0.03 ms of a 7B step). */
 enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2, SPEC_OPT_TRACE = 3,
-       SPEC_OPT_SMALL_GEMM_CTAS = 4, SPEC_OPT_GRAPH = 5 };
+       SPEC_OPT_SMALL_GEMM_CTAS = 4, SPEC_OPT_GRAPH = 5, SPEC_OPT_PHASE_TIMING = 6 };
 int spec_set_option(spec_ctx *ctx, int32_t what, int32_t value);
 
 /* Device timeline of the LAST step, recorded while SPEC_OPT_TRACE is on: one record per kernel
@@ -179,7 +181,8 @@ int spec_trace_read(spec_ctx *ctx, int32_t max_records, char *names, uint64_t *s
 /* Device time of the five parts of the LAST step, in milliseconds, from events recorded on
  * the stream at the part boundaries: ms[0] heads + lm_head + top-k, ms[1] tree expansion and
  * embedding gather, ms[2] verification forward incl. lm_head, ms[3] acceptance, ms[4] KV
- * compaction (the five parts of the step in Sec. III-B). Synchronises. */
+ * compaction (the five parts of the step in Sec. III-B). Needs SPEC_OPT_PHASE_TIMING on during that
+ * step (SPEC_E_STATE otherwise). Synchronises. */
 int spec_last_step_phase_ms(spec_ctx *ctx, float *ms /* HOST [5] */);
 
 /* Per-launch timing of one kernel kind of the verification forward: while `kind` != 0 every

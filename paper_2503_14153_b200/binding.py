@@ -20,7 +20,7 @@ FLAG_PACKED_WEIGHTS = 4
 PROFILE_OFF, PROFILE_GATE_UP, PROFILE_QKV, PROFILE_WO, PROFILE_DOWN, PROFILE_ATTENTION = range(6)
 
 Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB, Q_GRAPH_CAPTURES = 0, 1, 2, 3, 4, 5
-OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH, OPT_TRACE, OPT_SMALL_GEMM_CTAS, OPT_GRAPH = 0, 1, 2, 3, 4, 5
+OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH, OPT_TRACE, OPT_SMALL_GEMM_CTAS, OPT_GRAPH, OPT_PHASE_TIMING = 0, 1, 2, 3, 4, 5, 6
 TRACE_NAME_LEN = 32
 (DBG_TOK, DBG_POS, DBG_LOGITS, DBG_HIDDEN, DBG_ARGMAX, DBG_PATH, DBG_CAND, DBG_SEQLEN, DBG_NEXT_ROOT,
  DBG_H_LAST, DBG_STATUS) = range(11)

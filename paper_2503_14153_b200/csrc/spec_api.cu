@@ -246,6 +246,7 @@ struct spec_ctx {
   bool n_copy_pending = false;
   int n_copy_steps_after = 0;          // steps enqueued after the pending copy
   bool phase_valid = false;
+  bool phase_timing = false;           // SPEC_OPT_PHASE_TIMING
   int profile_kind = 0;                 // SPEC_PROFILE_*
   std::vector<cudaEvent_t> prof_ev;     // pairs, reused every step
   int prof_used = 0;
@@ -802,8 +803,10 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
   return SPEC_OK;
 }
 
-// Phase boundary i of the step: an event record (an external-event node while the step is being captured).
+// Phase boundary i of the step (only with SPEC_OPT_PHASE_TIMING: an event between two kernels costs the
+// programmatic overlap of that pair): an event record, an external-event node while the step is captured.
 void step_event(spec_ctx* c, int i) {
+  if (!c->phase_timing) return;
   if (c->capturing) cudaEventRecordWithFlags(c->phase_ev[i], c->stream, cudaEventRecordExternal);
   else cudaEventRecord(c->phase_ev[i], c->stream);
 }
@@ -932,7 +935,7 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     CUDA_OK(cudaGraphLaunch(g.exec, c->stream));
     c->launches += g.n_launches;
   }
-  c->phase_valid = true;
+  c->phase_valid = c->phase_timing;
   if (c->profile_kind) {
     CUDA_OK(cudaStreamSynchronize(c->stream));
     for (int i = 0; i + 1 < c->prof_used; i += 2) {
@@ -1155,6 +1158,8 @@ int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
   switch (what) {
     case SPEC_OPT_GRAPH:
       c->graph_on = value != 0; return SPEC_OK;
+    case SPEC_OPT_PHASE_TIMING:
+      c->phase_timing = value != 0; c->phase_valid = false; return SPEC_OK;
     case SPEC_OPT_PDL: c->pdl = value != 0; return SPEC_OK;
     case SPEC_OPT_GEMM_CTAS:
       if (value < 1 || value > SM_SLOTS) return c->fail(SPEC_E_BADARG, "gemm CTA count out of range");
@@ -1194,7 +1199,7 @@ int spec_trace_read(spec_ctx* c, int32_t max_records, char* names, uint64_t* sta
 
 int spec_last_step_phase_ms(spec_ctx* c, float* ms) {
   if (!c || !ms) return SPEC_E_BADARG;
-  if (!c->phase_valid) return c->fail(SPEC_E_STATE, "no step has run");
+  if (!c->phase_valid) return c->fail(SPEC_E_STATE, "no step has run with SPEC_OPT_PHASE_TIMING on");
   CUDA_OK(cudaStreamSynchronize(c->stream));
   for (int i = 0; i < 5; ++i) CUDA_OK(cudaEventElapsedTime(&ms[i], c->phase_ev[i], c->phase_ev[i + 1]));
   return SPEC_OK;

@@ -241,6 +241,13 @@ def test_timeline_and_options(torch):
         dec.set_option(99, 1)
     with pytest.raises(SpecError):
         dec.trace()                                     # tracing is off
+    with pytest.raises(SpecError):
+        dec.phase_ms()                                  # phase timing is off
+    dec.set_option(B.OPT_PHASE_TIMING, 1)
+    dec.step()
+    ph = dec.phase_ms()
+    assert ph.shape == (5,) and (ph > 0).all() and ph[2] == ph.max()   # the verification forward dominates
+    dec.set_option(B.OPT_PHASE_TIMING, 0)
     dec.set_option(B.OPT_TRACE, 1)
     l0 = dec.query(B.Q_KERNEL_LAUNCHES)
     dec.step()
