@@ -33,6 +33,7 @@ thread_local std::string g_create_error = "no error";
 constexpr int PREFILL_ROWS = 128;   // rows per sequence in one prefill pass
 constexpr int TRACE_CAP = 1024;     // launches of one step the timeline can hold
 constexpr int SM_SLOTS = 296;       // 148 SMs x 2 co-resident GEMM CTAs
+constexpr int N_COPY_EVERY = 4;         // enqueue-only steps between two copies of the committed lengths to the host
 constexpr int MAX_STEPS_AHEAD = 8;      // enqueue-only steps the host may run ahead of the device
 constexpr int ATTN_ROWS_WARPS = 6;      // warps of the CTA-per-16-rows attention kernel
 constexpr int ATTN_SPLIT_TILES = 8;       // fewest KV tiles a split of attention_tc gets (2..8 measured alike)
@@ -245,6 +246,7 @@ struct spec_ctx {
   cudaEvent_t n_ev = nullptr;
   bool n_copy_pending = false;
   int n_copy_steps_after = 0;          // steps enqueued after the pending copy
+  int steps_since_n_copy = 0;          // enqueue-only steps since the last copy was issued
   bool phase_valid = false;
   bool phase_timing = false;           // SPEC_OPT_PHASE_TIMING
   int profile_kind = 0;                 // SPEC_PROFILE_*
@@ -968,7 +970,9 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
           c->n_copy_pending = false;
         }
       }
-      if (!c->n_copy_pending &&
+      // a copy between two steps costs the overlap of the step's last kernel with the next step's first:
+      // one every N_COPY_EVERY steps keeps the bounds tight enough
+      if (!c->n_copy_pending && ++c->steps_since_n_copy >= N_COPY_EVERY && (c->steps_since_n_copy = 0, true) &&
           cudaMemcpyAsync(c->h_n_pinned, c->d_n, (size_t)B * sizeof(int), cudaMemcpyDeviceToHost, c->stream) == cudaSuccess &&
           cudaEventRecord(c->n_ev, c->stream) == cudaSuccess) {
         c->n_copy_pending = true;
