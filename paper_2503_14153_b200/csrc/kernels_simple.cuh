@@ -417,6 +417,17 @@ __global__ void __launch_bounds__(256) accept_kernel(AcceptArgs a, unsigned long
     return;
   }
   const int cnt = a.rows.cnt[b], m0 = b * R;
+  if (a.ntile <= 4) {
+    // few partial results per row: a thread per row, every row's loads in one trip
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+      float bv = -INFINITY; int bi = 0x7fffffff;
+      for (int t = 0; t < a.ntile; ++t) {
+        const float v = a.pval[(size_t)(m0 + i) * a.ntile + t]; const int idx = a.pidx[(size_t)(m0 + i) * a.ntile + t];
+        if (better(v, idx, bv, bi)) { bv = v; bi = idx; }
+      }
+      am_s[i] = bi; a.am[m0 + i] = bi;
+    }
+  } else
   for (int i = warp; i < cnt; i += nw) {
     float bv = -INFINITY; int bi = 0x7fffffff;
     const float* pv = a.pval + (size_t)(m0 + i) * a.ntile;
