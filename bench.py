@@ -327,7 +327,7 @@ def main():
                                "frac": gate_up_b / per / 1e9 / peak,
                                # dram__bytes_read.sum + dram__bytes_write.sum of this kernel at this shape
                                # (profiles/gemm_stream_7b_shapes_ncu_full.md); null for other shapes
-                               "traffic": 188.0e6 if (cfg.d_model, cfg.d_ffn, T) == (4096, 11008, 64) else None,
+                               "traffic": 186.5e6 if (cfg.d_model, cfg.d_ffn, T) == (4096, 11008, 64) else None,
                                "peak_kind": peak_kind,
                                "launches_timed": int(k_n), "us_per_launch": per * 1e6,
                                "algorithmic_bytes_per_launch": gate_up_b}
