@@ -648,56 +648,57 @@ __global__ void medusa_lmhead_topk(const T* __restrict__ r, const T* __restrict_
 
 // Merges the partial lists of one (sequence, head) row into cand[b][k+1][0..kmax) and applies
 // the optional override table; block 0 of each sequence also writes cand[b][0][0] = root.
-// Every slice's list is already ordered (value desc, index asc), so the row's best kmax are
-// found by a tournament over the list heads: one warp, each lane looking after every 32nd list.
-// Dynamic shared memory: nblocks * kmax * 8 + nblocks * 4 bytes.
-__global__ void topk_merge(const float* __restrict__ pk_val, const int* __restrict__ pk_idx, int nblocks,
-                           int rows_total, int K, int kmax, const int* __restrict__ root_tok,
-                           const int* __restrict__ cand_override, int* __restrict__ cand, unsigned long long* tr) {
+// The row's nblocks * kmax candidates sit in shared memory, every thread looking after each
+// blockDim-th of them; kmax rounds of a block-wide argmax (value desc, index asc), the owner of
+// the winner taking it out. Dynamic shared memory: nblocks * kmax * 8 bytes. At most 8 warps.
+__global__ void __launch_bounds__(256)
+topk_merge(const float* __restrict__ pk_val, const int* __restrict__ pk_idx, int nblocks,
+           int rows_total, int K, int kmax, const int* __restrict__ root_tok,
+           const int* __restrict__ cand_override, int* __restrict__ cand, unsigned long long* tr) {
   KTrace kt(tr);
   pdl_launch_dependents();
   pdl_wait();
   if (threadIdx.x == 0) trace_mark_min(tr, 2);
-  extern __shared__ float ms[];     // values [nblocks*kmax], indices [nblocks*kmax], list positions [nblocks]
-  int row = blockIdx.x, b = row / K, k = row % K;
-  int total = nblocks * kmax;
+  extern __shared__ float ms[];     // values [nblocks*kmax], indices [nblocks*kmax]
+  __shared__ float wv[8];
+  __shared__ int wi[8], wc[8];
+  const int row = blockIdx.x, b = row / K, k = row % K;
+  const int total = nblocks * kmax;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
   float* v = ms;
   int* ix = reinterpret_cast<int*>(ms + total);
-  int* head = ix + total;
   for (int c = threadIdx.x; c < total; c += blockDim.x) {
-    size_t o = (size_t)row * total + c;          // lists of a row are contiguous: [row][block][kmax]
+    const size_t o = (size_t)row * total + c;          // lists of a row are contiguous: [row][block][kmax]
     v[c] = pk_val[o];
     ix[c] = pk_idx[o];
   }
-  for (int c = threadIdx.x; c < nblocks; c += blockDim.x) head[c] = 0;
+  // the override entries do not depend on the lists: one load per round, issued up front
+  int ovr = -1;
+  if (cand_override && threadIdx.x < kmax) ovr = cand_override[((size_t)b * K + k) * kmax + threadIdx.x];
   __syncthreads();
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    int* out = cand + ((size_t)b * (K + 1) + k + 1) * kmax;
-    for (int t = 0; t < kmax; ++t) {
-      float bv = -INFINITY; int bi = 0x7fffffff, bl = -1;
-      for (int l = lane; l < nblocks; l += 32) {
-        const int pos = head[l];
-        if (pos < kmax && better(v[l * kmax + pos], ix[l * kmax + pos], bv, bi)) { bv = v[l * kmax + pos]; bi = ix[l * kmax + pos]; bl = l; }
-      }
+  int* out = cand + ((size_t)b * (K + 1) + k + 1) * kmax;
+  for (int t = 0; t < kmax; ++t) {
+    float bv = -INFINITY; int bi = 0x7fffffff, bc = -1;
+    for (int c = threadIdx.x; c < total; c += blockDim.x)
+      if (better(v[c], ix[c], bv, bi)) { bv = v[c]; bi = ix[c]; bc = c; }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        int oi = __shfl_xor_sync(0xffffffffu, bi, o), ol = __shfl_xor_sync(0xffffffffu, bl, o);
-        if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bl = ol; }
-      }
-      // every lane now holds the winner; the lane that looks after its list moves that list on
-      if (bl >= 0 && (bl & 31) == lane) head[bl]++;
-      if (lane == 0) {
-        int tokv = bi;
-        if (cand_override) {
-          int o = cand_override[((size_t)b * K + k) * kmax + t];
-          if (o >= 0) tokv = o;
-        }
-        out[t] = (tokv == 0x7fffffff) ? 0 : tokv;
-      }
-      __syncwarp();
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o), oc = __shfl_xor_sync(0xffffffffu, bc, o);
+      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; bc = oc; }
     }
+    if (lane == 0) { wv[warp] = bv; wi[warp] = bi; wc[warp] = bc; }
+    __syncthreads();
+    bv = wv[0]; bi = wi[0]; bc = wc[0];
+    for (int w = 1; w < nw; ++w)
+      if (better(wv[w], wi[w], bv, bi)) { bv = wv[w]; bi = wi[w]; bc = wc[w]; }
+    // every thread holds the winner; its owner takes it out, thread t publishes rank t
+    if (bc >= 0 && bc % (int)blockDim.x == (int)threadIdx.x) { v[bc] = -INFINITY; ix[bc] = 0x7fffffff; }
+    if ((int)threadIdx.x == t) {
+      const int tokv = ovr >= 0 ? ovr : bi;
+      out[t] = (tokv == 0x7fffffff) ? 0 : tokv;
+    }
+    __syncthreads();
   }
   if (k == 0 && threadIdx.x == 0) cand[(size_t)b * (K + 1) * kmax] = root_tok[b];
 }
