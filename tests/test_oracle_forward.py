@@ -196,3 +196,75 @@ def test_bf16_mode_stays_close_to_exact():
     b = forward_full(OracleModel(cfg.with_(dtype="fp32"), wq), toks)
     assert np.abs(a - b).max() <= 2e-2 * np.abs(b).max()
     assert np.abs(a - b).max() > 0
+
+
+def _head_only_model(d, V, W, b, lm):
+    """An OracleModel that holds just one extra head and the lm_head (all medusa_logits reads)."""
+    cfg = SMALL.with_(d_model=d, vocab=V, n_medusa=1, topk=(1,), dtype="fp32")
+    return OracleModel(cfg, {"medusa.0.w": np.asarray(W, np.float32), "medusa.0.b": np.asarray(b, np.float32),
+                             "lm_head": np.asarray(lm, np.float32)})
+
+
+def test_medusa_head_hand_worked_2x2():
+    """Extra head on the last hidden state (Sec. III-B, model architecture): residual block
+    h + SiLU(W h + b) with W stored [out, in], then the shared lm_head. Worked by hand:
+    W = [[1, 2], [0, -1]], b = (0, 1), h = (1, 1): W h + b = (3, 0), SiLU -> (3 / (1 + e^-3), 0),
+    r = (1 + 3 / (1 + e^-3), 1); lm_head = [[0, 1], [1, 0], [1, 1]] -> z = (r1, r0, r0 + r1).
+    With W transposed W^T h + b = (1, 2) and z differs in every entry."""
+    m = _head_only_model(2, 3, [[1, 2], [0, -1]], [0, 1], [[0, 1], [1, 0], [1, 1]])
+    z = medusa_logits(m, np.array([1.0, 1.0]))
+    r0 = 1.0 + 3.0 / (1.0 + np.exp(-3.0))
+    assert np.allclose(z[0], [1.0, r0, r0 + 1.0], rtol=1e-6)
+
+
+def test_medusa_head_matches_torch_linear_modules():
+    """The same block written with torch.nn.Linear modules in float64 (weight [out, in], x W^T + b)
+    on a random, non-symmetric head matrix: a transposed matrix, a dropped bias or residual,
+    or the lm_head applied to the wrong vector fails."""
+    torch = pytest.importorskip("torch")
+    cfg = SMALL.with_(n_medusa=3, topk=(3, 2, 2))
+    w = draw_weights(cfg)
+    for k in range(3):                                   # N(0, 0.02) would make SiLU nearly linear: scale up
+        w[f"medusa.{k}.w"] = (w[f"medusa.{k}.w"] * 40.0).astype(np.float32)
+        w[f"medusa.{k}.b"] = (w[f"medusa.{k}.b"] * 20.0).astype(np.float32)
+    h = np.random.default_rng(12).standard_normal(cfg.d_model)
+    z = medusa_logits(OracleModel(cfg, w), h)
+    lm = torch.nn.Linear(cfg.d_model, cfg.vocab, bias=False, dtype=torch.float64)
+    th = torch.from_numpy(h)
+    with torch.no_grad():
+        lm.weight.copy_(torch.from_numpy(w["lm_head"]).double())
+        for k in range(3):
+            blk = torch.nn.Linear(cfg.d_model, cfg.d_model, bias=True, dtype=torch.float64)
+            blk.weight.copy_(torch.from_numpy(w[f"medusa.{k}.w"]).double())
+            blk.bias.copy_(torch.from_numpy(w[f"medusa.{k}.b"]).double())
+            ref = lm(th + torch.nn.functional.silu(blk(th))).numpy()
+            assert np.abs(z[k] - ref).max() <= 2e-6 * np.abs(ref).max()      # float32 rounding of z
+            wrong = lm(th + torch.nn.functional.silu(th @ blk.weight + blk.bias)).numpy()
+            assert np.abs(z[k] - wrong).max() > 1e-2 * np.abs(ref).max()     # the transposed reading is far away
+
+
+def test_prefill_across_chunk_boundaries_equals_full_forward():
+    """OracleSpecDecoder.prefill walks the prompt in chunks; a 150-token prompt in chunks of 32
+    (four full chunks and a ragged one) must leave the first root token, its logits and the
+    cache rows of the plain causal forward over the whole prompt."""
+    from oracle.spec import OracleSpecDecoder
+    from oracle.tree import build_tree
+    cfg = SMALL
+    m = OracleModel(cfg, draw_weights(cfg))
+    prompt = np.random.default_rng(13).integers(0, cfg.vocab, 150)
+    full = forward_full(m, prompt)
+    dec = OracleSpecDecoder(m, build_tree((2, 2, 2), 6), 200)
+    dec.prefill(prompt, chunk=32)
+    assert dec.n == 150
+    assert np.abs(dec.last_root_logits - full[-1]).max() <= 1e-6 * np.abs(full[-1]).max()
+    assert dec.root_tok == int(np.argmax(full[-1].astype(np.float32)))
+    # a later row sees every earlier chunk: the next token's logits after one more cached row
+    one = KVCache(cfg, 151)
+    forward_rows(m, one, 0, prompt, np.arange(150), np.tril(np.ones((150, 150), bool)))
+    for l in range(cfg.n_layers):
+        assert np.allclose(dec.cache.k[l, :150], one.k[l, :150], atol=1e-12)
+        assert np.allclose(dec.cache.v[l, :150], one.v[l, :150], atol=1e-12)
+    ext = np.concatenate([prompt, [dec.root_tok]])
+    _, lg = forward_rows(m, dec.cache, 150, [dec.root_tok], [150], np.ones((1, 1), bool))
+    ref = forward_full(m, ext)[-1]
+    assert np.abs(lg[0] - ref).max() <= 1e-6 * np.abs(ref).max()

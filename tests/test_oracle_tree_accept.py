@@ -157,3 +157,22 @@ def test_fragment_truncation_rule():
     assert truncate_to_fragment([5, 9, 5, 9], 9) == 4
     assert truncate_to_fragment([5, 6, 7], 9) == 1      # no marker: keep the root only
     assert truncate_to_fragment([9, 6, 7], 9) == 1
+
+
+def test_typical_accept_temperature_two_token_closed_form():
+    """Eq. 1 with p = softmax(logits / temperature) on a two-token vocabulary. Root logits
+    (temperature * ln 3, 0) give p = (3/4, 1/4) at every temperature, H = ln 4 - (3/4) ln 3 and
+    exp(-H) = 3^(3/4) / 4 = 0.56988; with eps = 1 the threshold is delta * 0.56988: 0.2849 at
+    delta 0.5 and 0.2279 at delta 0.4. The child carries token 1 (p = 1/4), so it is rejected
+    at delta 0.5 and accepted at delta 0.4, whatever the temperature. A rule that multiplied
+    the logits by the temperature would see p = (0.568, 0.432) at temperature 0.5 (accepts at
+    delta 0.5) and p = (81/82, 1/82) at temperature 2 (rejects at delta 0.4)."""
+    assert 3 ** 0.75 / 4 == pytest.approx(0.5698768, abs=1e-6)
+    parent, depth, tok = np.array([-1, 0]), np.array([0, 1]), np.array([0, 1])
+    for temperature in (0.5, 1.0, 2.0):
+        lg = np.zeros((2, 2))
+        lg[0] = [temperature * np.log(3.0), 0.0]
+        assert typical_accept(parent, depth, tok, lg, 1.0, 0.5, temperature) == [0]
+        assert typical_accept(parent, depth, tok, lg, 1.0, 0.4, temperature) == [0, 1]
+        # eps is the smaller bound: 0.2 < 0.2849 lets the p = 1/4 token through
+        assert typical_accept(parent, depth, tok, lg, 0.2, 0.5, temperature) == [0, 1]
