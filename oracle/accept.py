@@ -67,6 +67,18 @@ def typical_accept(parent, depth, tok, logits, eps: float, delta: float, tempera
     return select_path(parent, depth, edge)
 
 
+def sample_token(logits, temperature: float, u: float) -> int:
+    """Sampled decoding at a temperature: the token drawn from softmax(logits / temperature) by
+    inverting the cumulative distribution in token order at the uniform u in [0, 1): the first
+    token j whose cumulative weight sum_{i <= j} exp((z_i - max z) / temperature) exceeds
+    u times the total weight."""
+    z = np.asarray(logits, dtype=np.float64) / temperature
+    w = np.exp(z - z.max())
+    cdf = np.cumsum(w)
+    j = int(np.searchsorted(cdf, u * cdf[-1], side="right"))
+    return min(j, len(w) - 1)
+
+
 def truncate_to_fragment(path_tokens, frag_token: int) -> int:
     """Fragment-integrity rule of Sec. III-B: keep the accepted span up to and including
     its last fragment marker; with no marker in the span only the first token is kept.

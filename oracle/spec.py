@@ -8,8 +8,9 @@ become the next cached positions.
 """
 import numpy as np
 
-from .accept import argmax_lowest, greedy_accept, truncate_to_fragment, typical_accept
+from .accept import argmax_lowest, greedy_accept, sample_token, truncate_to_fragment, typical_accept
 from .decoder import KVCache, OracleModel, forward_full, forward_rows, medusa_logits, top_k
+from .rng import step_uniform
 from .tree import ancestor_mask
 
 
@@ -28,7 +29,7 @@ def greedy_decode_nocache(model: OracleModel, prompt, new_tokens: int) -> np.nda
 class OracleSpecDecoder:
     def __init__(self, model: OracleModel, tree, max_seq: int, accept_mode: str = "greedy",
                  typ_eps: float = 0.09, typ_delta: float = 0.3, temperature: float = 1.0,
-                 frag_token: int = -1):
+                 frag_token: int = -1, sampling: bool = False, seed: int = 0, sequence: int = 0):
         self.model, self.cfg = model, model.cfg
         self.parent = np.asarray(tree["parent"], dtype=np.int32)
         self.depth = np.asarray(tree["depth"], dtype=np.int32)
@@ -39,6 +40,10 @@ class OracleSpecDecoder:
         self.accept_mode = accept_mode
         self.typ = (typ_eps, typ_delta, temperature)
         self.frag_token = frag_token
+        # sampled decoding (Sec. IV-B times every prompt greedy and at temperature 0.8): the token that
+        # follows the accepted span is drawn from softmax(logits / temperature) instead of the argmax
+        self.sampling, self.seed, self.sequence = sampling, seed, sequence
+        self.draws = 0                      # draw counter: 0 for the token after the prompt, then one per step
         self.n = 0
         self.root_tok = None
         self.h_last = None
@@ -56,8 +61,17 @@ class OracleSpecDecoder:
                                           np.tril(np.ones((c, c), dtype=bool)), [c - 1])
             self.n += c
         self.h_last = hidden[-1]
-        self.root_tok = int(argmax_lowest(logits[0]))
+        self.draws = 0
+        self.root_tok = self._next_token(logits[0])
         self.last_root_logits = logits[0]
+
+    def _next_token(self, logits_row) -> int:
+        """Base model's own next token: the argmax, or in sampled decoding the draw at this step's uniform."""
+        if not self.sampling:
+            return int(argmax_lowest(logits_row))
+        self.last_u = step_uniform(self.seed, self.sequence, self.draws)
+        self.draws += 1
+        return sample_token(logits_row, self.typ[2], self.last_u)
 
     def candidates(self):
         """cand[0][0] = root token; cand[k][j] = j-th best token of head k."""
@@ -90,12 +104,13 @@ class OracleSpecDecoder:
             self.cache.k[l, self.n:self.n + count] = self.cache.k[l, self.n + np.asarray(path)]
             self.cache.v[l, self.n:self.n + count] = self.cache.v[l, self.n + np.asarray(path)]
         best = path[-1]
+        next_root = self._next_token(logits[best])
         rec = {"cand": cand, "head_logits": z, "tok": tok, "pos": pos, "logits": logits,
                "hidden": hidden, "am": am, "path": np.asarray(path, dtype=np.int32),
                "count": count, "tokens": tok[path].astype(np.int32), "n_before": self.n,
-               "next_root": int(am[best])}
+               "next_root": next_root, "best": int(best)}
         self.n += count
-        self.root_tok = int(am[best])
+        self.root_tok = next_root
         self.h_last = hidden[best]
         return rec
 
