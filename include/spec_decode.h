@@ -59,6 +59,10 @@ typedef struct {
   float typ_eps, typ_delta, temperature; /* Eq. 1 hyper-parameters; softmax temperature   */
   int32_t frag_token;   /* fragment marker id for the fragment-integrity rule; -1 = off   */
   int32_t flags;        /* SPEC_FLAG_* bits                                               */
+  int32_t sampling;     /* 0 = the token that follows the accepted span is the base model's
+                           argmax there; 1 = sampled decoding (Sec. IV-B): it is drawn from
+                           softmax(logits / temperature) (needs accept_mode 1, temperature > 0) */
+  uint32_t seed_lo, seed_hi; /* 64-bit seed of the sampler's counter-based generator        */
 } spec_config;
 
 #define SPEC_FLAG_KEEP_LOGITS 1 /* materialise verify logits [rows, vocab] for spec_debug_read  */
@@ -129,7 +133,13 @@ int spec_prefill(spec_ctx *ctx, int32_t batch, const int32_t *tokens, const int3
  * after they are valid. If both are NULL the step is only enqueued on the stream (no host
  * synchronisation); emitted tokens are then read later with spec_read_generated.
  * cand_override: optional HOST table [batch][n_medusa][kmax] (kmax = spec_query(SPEC_Q_KMAX));
- * an entry >= 0 replaces that head candidate after the heads have run, -1 keeps it. */
+ * an entry >= 0 replaces that head candidate after the heads have run, -1 keeps it.
+ * Sampled decoding (spec_config.sampling): the token after the accepted span -- the next step's
+ * root -- is the first token j whose cumulative weight sum_{i<=j} exp((z_i - max z) / temperature)
+ * exceeds u times the total, z the last accepted node's logits (double precision sums in token
+ * order), u = (w >> 8) * 2^-24 with w the first output word of Philox-4x32-10 at counter
+ * (draw index, sequence, 0, 0) and key (seed_lo, seed_hi); draw 0 is the token after the prompt
+ * (spec_prefill), every step takes the next one. */
 int spec_step(spec_ctx *ctx, int32_t *out_tokens, int32_t *out_counts, const int32_t *cand_override);
 
 /* Copies up to `max_tokens` tokens generated so far by sequence `seq` (all steps since
@@ -145,7 +155,8 @@ const char *spec_last_error(const spec_ctx *ctx);
 /* Integer properties of a context. */
 enum { SPEC_Q_KMAX = 0, SPEC_Q_KERNEL_LAUNCHES = 1, SPEC_Q_N_NODES = 2, SPEC_Q_BATCH = 3,
        SPEC_Q_ALGO_BYTES_PER_STEP = 4 /* weights + lm_head (twice) + heads, in KiB */,
-       SPEC_Q_GRAPH_CAPTURES = 5 /* times a step was recorded into a CUDA graph */ };
+       SPEC_Q_GRAPH_CAPTURES = 5 /* times a step was recorded into a CUDA graph */,
+       SPEC_Q_CLUSTER_GATE_UP = 6 /* 1 if a step's gate+up projection runs as the cluster kernel with the SwiGLU inside */ };
 int64_t spec_query(const spec_ctx *ctx, int32_t what);
 
 /* Tuning knobs of a context (defaults in brackets). SPEC_OPT_PDL [1]: launch the kernels of
@@ -164,9 +175,19 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
  * after a prefill and after an option change; steps that are traced or profiled are enqueued
  * directly). Results do not depend on it. SPEC_OPT_PHASE_TIMING [0]: record an event at the five
  * phase boundaries of every step for spec_last_step_phase_ms (costs the programmatic overlap at
- * those boundaries: about 0.03 ms of a 7B step). */
+ * those boundaries: about 0.03 ms of a 7B step). SPEC_OPT_CLUSTER_EPILOGUE [2]: bit mask of the projections
+ * that, in passes of at most 128 rows, run as thread-block clusters which add their split-K sums through
+ * distributed shared memory and apply the step that follows themselves: 1 = output and down projections
+ * (residual add in place), 2 = gate+up (SwiGLU, passes of at most 64 rows), 4 = q/k/v (RoPE and cache
+ * store). A projection whose bit is clear leaves partial sums for a separate kernel (other summation
+ * order, same rounding points). Only bit 2 is on by default: on the 7B shape it is the one that is
+ * faster (bits 1 and 4 cost 2% and 4% of a step there). SPEC_OPT_WIDE_GEMM [1]: passes of more than
+ * 128 rows (batched verification, batched prompt processing) run their projections as whole
+ * [128 weight rows] x [256 activation rows] tiles that keep a weight tile for 256 rows at a time;
+ * 0 = the weight-streaming kernel, which re-reads the weights for every 128 rows. */
 enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2, SPEC_OPT_TRACE = 3,
-       SPEC_OPT_SMALL_GEMM_CTAS = 4, SPEC_OPT_GRAPH = 5, SPEC_OPT_PHASE_TIMING = 6 };
+       SPEC_OPT_SMALL_GEMM_CTAS = 4, SPEC_OPT_GRAPH = 5, SPEC_OPT_PHASE_TIMING = 6, SPEC_OPT_CLUSTER_EPILOGUE = 7,
+       SPEC_OPT_WIDE_GEMM = 8 };
 int spec_set_option(spec_ctx *ctx, int32_t what, int32_t value);
 
 /* Device timeline of the LAST step, recorded while SPEC_OPT_TRACE is on: one record per kernel
@@ -214,6 +235,13 @@ int spec_debug_read(spec_ctx *ctx, int32_t what, void *host_buf, size_t bytes);
  * to HOST float32 arrays [n_slots][n_kv_heads][head_dim] in logical (unpaged) order. */
 int spec_debug_read_kv(spec_ctx *ctx, int32_t seq, int32_t layer, int32_t slot0, int32_t n_slots,
                        float *host_k, float *host_v);
+
+/* Self test of the bounded device-side waits (SPEC_E_TIMEOUT). Every wait of the library's kernels on an
+ * mbarrier gives up after a time limit, records ST_TIMEOUT and the place in the device status word and lets
+ * the kernel return; the host then reports SPEC_E_TIMEOUT. This entry runs one warp that waits, with a limit
+ * of limit_us microseconds (1..100000), on a barrier nothing completes: it returns SPEC_E_TIMEOUT (and
+ * spec_last_error names place 99), clears the status word, and the context remains usable. Synchronises. */
+int spec_debug_wait_timeout(spec_ctx *ctx, int32_t limit_us);
 
 /* ---- single operations of the verify forward, for unit parity tests and profiling ---- */
 
@@ -263,7 +291,8 @@ int spec_build_labels(const int32_t *tokens, int32_t n_seq, int32_t seq_len, int
  * The partial sums and the status word live in an array built into the library
  * (SPEC_STATIC_SCRATCH_FLOATS float32 values, 8 MiB, held by every GPU that loads the library
  * until the process exits). A call that needs more than that (spec_op_linear_scratch_floats()
- * says how much a shape needs) returns SPEC_E_NOMEM and spec_last_error(NULL) says by how much. The call itself allocates nothing, on host or device.
+ * says how much a shape needs) returns SPEC_E_NOMEM and spec_last_error(NULL) says by how much. A call that
+ * succeeds allocates nothing, on host or device (a failing one builds its error text on the host).
  * The first call on each device looks the array's device address up (with that device
  * current) and keeps it; make that first call outside any stream capture. All calls share the
  * one array: it still holds the previous call's partial sums (the library clears the status

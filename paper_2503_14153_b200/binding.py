@@ -19,8 +19,8 @@ FLAG_SIMPLE_KERNELS = 2
 FLAG_PACKED_WEIGHTS = 4
 PROFILE_OFF, PROFILE_GATE_UP, PROFILE_QKV, PROFILE_WO, PROFILE_DOWN, PROFILE_ATTENTION = range(6)
 
-Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB, Q_GRAPH_CAPTURES = 0, 1, 2, 3, 4, 5
-OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH, OPT_TRACE, OPT_SMALL_GEMM_CTAS, OPT_GRAPH, OPT_PHASE_TIMING = 0, 1, 2, 3, 4, 5, 6
+Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB, Q_GRAPH_CAPTURES, Q_CLUSTER_GATE_UP = 0, 1, 2, 3, 4, 5, 6
+OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH, OPT_TRACE, OPT_SMALL_GEMM_CTAS, OPT_GRAPH, OPT_PHASE_TIMING, OPT_CLUSTER_EPILOGUE, OPT_WIDE_GEMM = 0, 1, 2, 3, 4, 5, 6, 7, 8
 TRACE_NAME_LEN = 32
 (DBG_TOK, DBG_POS, DBG_LOGITS, DBG_HIDDEN, DBG_ARGMAX, DBG_PATH, DBG_CAND, DBG_SEQLEN, DBG_NEXT_ROOT,
  DBG_H_LAST, DBG_STATUS) = range(11)
@@ -29,7 +29,7 @@ EXPORTS = ["spec_workspace_bytes", "spec_create", "spec_prefill", "spec_step", "
            "spec_destroy", "spec_last_error", "spec_query", "spec_debug_read", "spec_debug_read_kv",
            "spec_op_linear", "spec_op_linear_scratch_floats", "spec_op_linear_static", "spec_packed_weight_bytes",
            "spec_pack_weight", "spec_set_option", "spec_trace_read", "spec_build_labels", "spec_last_step_phase_ms", "spec_profile_kernel",
-           "spec_profile_read"]
+           "spec_profile_read", "spec_debug_wait_timeout"]
 
 
 class SpecError(RuntimeError):
@@ -43,7 +43,8 @@ class SpecConfig(C.Structure):
                [("rms_eps", C.c_float), ("rope_base", C.c_float), ("dtype", C.c_int32), ("n_medusa", C.c_int32),
                 ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("page_size", C.c_int32), ("accept_mode", C.c_int32),
                 ("typ_eps", C.c_float), ("typ_delta", C.c_float), ("temperature", C.c_float),
-                ("frag_token", C.c_int32), ("flags", C.c_int32)]
+                ("frag_token", C.c_int32), ("flags", C.c_int32), ("sampling", C.c_int32),
+                ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32)]
 
 
 class SpecTree(C.Structure):
@@ -113,6 +114,8 @@ def load_library():
     lib.spec_pack_weight.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     lib.spec_last_step_phase_ms.restype = C.c_int
     lib.spec_last_step_phase_ms.argtypes = [C.c_void_p, C.c_void_p]
+    lib.spec_debug_wait_timeout.restype = C.c_int
+    lib.spec_debug_wait_timeout.argtypes = [C.c_void_p, C.c_int32]
     lib.spec_profile_kernel.restype = C.c_int
     lib.spec_profile_kernel.argtypes = [C.c_void_p, C.c_int32]
     lib.spec_profile_read.restype = C.c_int
@@ -199,7 +202,7 @@ class SpecDecoder:
     def __init__(self, cfg, dev_weights: Dict[str, "object"], tree: Dict[str, np.ndarray], max_seq: int,
                  max_batch: int = 1, flags: int = 0, accept_mode: int = 0, typ_eps: float = 0.09,
                  typ_delta: float = 0.3, temperature: float = 1.0, frag_token: int = -1, stream=None,
-                 packed: Optional[bool] = None):
+                 packed: Optional[bool] = None, sampling: bool = False, seed: int = 0):
         import torch
         tc_path = cfg.dtype == "bf16" and not (flags & FLAG_SIMPLE_KERNELS)
         self.packed = tc_path if packed is None else bool(packed)
@@ -221,7 +224,7 @@ class SpecDecoder:
         self._ccfg = SpecConfig(cfg.n_layers, cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim, cfg.d_ffn,
                                 cfg.vocab, cfg.rms_eps, cfg.rope_base, 1 if cfg.dtype == "bf16" else 0, cfg.n_medusa,
                                 max_batch, max_seq, cfg.page_size, accept_mode, typ_eps, typ_delta, temperature,
-                                frag_token, flags)
+                                frag_token, flags, 1 if sampling else 0, seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
         L = cfg.n_layers
         qrows = cfg.n_heads * cfg.head_dim
         krows = cfg.n_kv_heads * cfg.head_dim
@@ -346,8 +349,17 @@ class SpecDecoder:
             out.append((nm,) + tuple(int(v) for v in stamps[i]))
         return out
 
+    def wait_timeout_probe(self, limit_us: int) -> int:
+        """Runs the bounded-wait self test; returns the library's code (SPEC_E_TIMEOUT = -6 when it works)."""
+        return int(self.lib.spec_debug_wait_timeout(self._ctx, limit_us))
+
     def set_option(self, what: int, value: int):
         self._check(self.lib.spec_set_option(self._ctx, what, value))
+
+    def gate_up_kernel_name(self) -> str:
+        """Name of the kernel a step's gate+up projection runs as (the dominant kernel of a 7B step)."""
+        mt = 16 if self.batch * self.T <= 16 else (32 if self.batch * self.T <= 32 else (64 if self.batch * self.T <= 64 else 128))
+        return f"gemm_cluster<{mt},swiglu>" if self.query(Q_CLUSTER_GATE_UP) else f"gemm_stream<{mt}>"
 
     def query(self, what: int) -> int:
         return int(self.lib.spec_query(self._ctx, what))

@@ -119,14 +119,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after ~2 s, records where in the status word and returns false.
+// Bounded wait: gives up after limit_ns (2 s unless the caller says otherwise), records where in the
+// status word and returns false.
 #define SPEC_WAIT_LIMIT_NS 2000000000ull
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int where) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int where,
+                                          uint64_t limit_ns = SPEC_WAIT_LIMIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
   uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 0x3ff) == 0 && global_timer_ns() - t0 > SPEC_WAIT_LIMIT_NS) {
+    if ((++spins & 0x3f) == 0 && global_timer_ns() - t0 > limit_ns) {
       set_status(status, ST_TIMEOUT, where, (int)parity);
       return false;
     }

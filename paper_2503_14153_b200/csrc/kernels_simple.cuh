@@ -370,6 +370,105 @@ __global__ void typical_edges(const float* __restrict__ logits, int V, Rows rows
   }
 }
 
+// ------------------------------------------------------------------ sampled decoding
+// Philox-4x32, 10 rounds (Salmon et al., SC 2011): counter c[4], key k[2] -> four 32-bit words.
+__device__ __forceinline__ void philox4x32_10(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    if (r) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c[0]), lo0 = 0xD2511F53u * c[0];
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c[2]), lo1 = 0xCD9E8D57u * c[2];
+    const uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
+    c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
+  }
+}
+
+// Sampled decoding at a temperature (Sec. IV-B: every prompt is also decoded by sampling): the
+// token that follows the accepted span is drawn from softmax(logits / temperature) of the last
+// accepted node by inverting the cumulative distribution in token order at the uniform
+// u = top 24 bits of philox(counter = (draw index, sequence, 0, 0), key = seed) * 2^-24.
+// One block per sequence; thread t owns a contiguous chunk of the vocabulary, the chunks' weights
+// are summed in double precision, a prefix over the chunks finds the chunk that holds u * total
+// and its owner scans it. prefill != 0: the row is the sequence's last prompt position (row b).
+__global__ void __launch_bounds__(256)
+sample_root(const float* __restrict__ logits, int V, int R, int K, const int* __restrict__ path,
+            const int* __restrict__ count, float temperature, uint32_t seed_lo, uint32_t seed_hi,
+            int* __restrict__ draws, int* __restrict__ root_tok, int prefill) {
+  const int b = blockIdx.x;
+  int row = b;
+  if (!prefill) {
+    const int len = count[b];
+    if (len < 1) return;
+    row = b * R + path[b * (K + 1) + len - 1];
+  }
+  const float* z = logits + (size_t)row * V;
+  const double inv_t = 1.0 / (double)temperature;
+  __shared__ double red[256];
+  __shared__ double mx_s;
+  __shared__ int chunk_s;
+  __shared__ double target_s, before_s;
+  const int per = (V + blockDim.x - 1) / blockDim.x;
+  const int c0 = threadIdx.x * per, c1 = min(V, c0 + per);
+  double mx = -INFINITY;
+  for (int c = c0; c < c1; ++c) mx = fmax(mx, (double)z[c] * inv_t);
+  red[threadIdx.x] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double m = -INFINITY;
+    for (int t = 0; t < (int)blockDim.x; ++t) m = fmax(m, red[t]);
+    mx_s = m;
+  }
+  __syncthreads();
+  mx = mx_s;
+  double sum = 0.0;
+  for (int c = c0; c < c1; ++c) sum += exp((double)z[c] * inv_t - mx);
+  __syncthreads();
+  red[threadIdx.x] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t ctr[4] = {(uint32_t)draws[b], (uint32_t)b, 0u, 0u};
+    philox4x32_10(ctr, seed_lo, seed_hi);
+    const double u = (double)(ctr[0] >> 8) * (1.0 / 16777216.0);
+    double total = 0.0;
+    for (int t = 0; t < (int)blockDim.x; ++t) total += red[t];
+    const double target = u * total;
+    // total was added in this order, so the last non-empty chunk always exceeds the target (u < 1)
+    double acc = 0.0;
+    int chunk = 0;
+    for (int t = 0; t < (int)blockDim.x; ++t) {
+      chunk = t;
+      if (acc + red[t] > target) break;
+      acc += red[t];
+    }
+    chunk_s = chunk; target_s = target; before_s = acc;
+    draws[b] += 1;
+  }
+  __syncthreads();
+  if ((int)threadIdx.x == chunk_s) {
+    // (the scan adds the chunk's weights one by one onto the prefix; should rounding keep it from
+    // passing the target, the chunk's last token is the answer)
+    double acc = before_s;
+    int pick = c1 - 1;
+    for (int c = c0; c < c1; ++c) {
+      acc += exp((double)z[c] * inv_t - mx);
+      if (acc > target_s) { pick = c; break; }
+    }
+    root_tok[b] = pick;
+  }
+}
+
+// ------------------------------------------------------------------ bounded-wait self test
+// One warp waits on an mbarrier that nothing will ever complete, with the given time limit: the wait
+// gives up, records ST_TIMEOUT with where = 99 in the status word and the kernel returns normally.
+__global__ void wait_probe(int* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+    mbar_wait(&bar, 0, status, 99, limit_ns);
+  }
+}
+
 // ------------------------------------------------------------------ acceptance walk
 struct AcceptArgs {
   Rows rows;

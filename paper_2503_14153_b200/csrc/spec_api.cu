@@ -19,7 +19,9 @@
 
 #include "attention_tc.cuh"
 #include "common.cuh"
+#include "gemm_cluster.cuh"
 #include "gemm_stream.cuh"
+#include "gemm_wide.cuh"
 #include "glue_tc.cuh"
 #include "kernels_simple.cuh"
 #include "labels.cuh"
@@ -144,9 +146,19 @@ int plan_slot_bound(const GemmPlan& g) {
 
 size_t plan_part_floats(const GemmPlan& g) { return (size_t)plan_slot_bound(g) * g.p.M * g.p.n_tiles * 128; }
 
+// The shared-memory attribute of a kernel is per device: it is set on every launch's device the first time
+// that device is seen (indexed by the device ordinal), not once per process.
+constexpr int kAttrDevices = 64;
+inline bool* attr_flag(bool (&flags)[kAttrDevices]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kAttrDevices) dev = 0;
+  return &flags[dev];
+}
+
 template <int MT, int DEEP>
 cudaError_t launch_gs_mt(cudaStream_t st, bool pdl, int grid, const StreamTmaps& tm, const StreamGemmParams& p) {
-  static bool attr_set = false;
+  static bool attr_set_dev[kAttrDevices] = {};
+  bool& attr_set = *attr_flag(attr_set_dev);
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(gemm_stream<MT, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamCfg<MT, DEEP>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
@@ -187,6 +199,10 @@ struct spec_ctx {
   bool pdl = true;                     // programmatic dependent launch between the kernels of a step
   int gemm_ctas = 288;                 // persistent CTAs of the weight-streaming GEMM (measured best; at most SM_SLOTS)
   int l2_prefetch = 0;
+  bool gc_attr_set[12] = {};            // per context (and so per device): shared-memory attribute of each gemm_cluster instance set
+  bool wide_gemm = true;               // SPEC_OPT_WIDE_GEMM: passes of more than 128 rows use the 128 x 256-tile kernel
+  int cluster_epilogue = 2;            // SPEC_OPT_CLUSTER_EPILOGUE: which projections finish their split-K sums inside a cluster
+                                       // (bits: 1 output/down, 2 gate+up, 4 q/k/v; measured on the 7B shape: only gate+up pays)
   int small_gemm_ctas = 288;           // CTAs of GEMMs with at most 48 weight tiles (Wo, down); 288 since the weights are pre-tiled (192 before)
   std::vector<int> h_parent, h_depth, h_rank;
   std::vector<int> n_hi, n_lo;         // host upper / lower bounds of the committed lengths
@@ -198,7 +214,7 @@ struct spec_ctx {
   // device buffers (workspace)
   int *d_n, *d_cnt, *d_n_old, *d_root, *d_count, *d_path, *d_out_tok, *d_gen_cnt, *d_gen_log, *d_cand, *d_cand_ov;
   int *d_tok, *d_pos, *d_slot, *d_am, *d_edge, *d_parent, *d_depth, *d_rank, *d_page_table, *d_prompt, *d_offsets;
-  int *d_status, *d_pidx, *d_pk_idx;
+  int *d_status, *d_pidx, *d_pk_idx, *d_draws;
   uint32_t *d_anc_tree, *d_anc_chain;
   const void **d_mw, **d_mb;
   float *d_x, *d_hid, *d_h_last, *d_part, *d_logits, *d_pval, *d_part_o, *d_part_ml, *d_pk_val;
@@ -296,6 +312,8 @@ bool validate_config(const spec_config* c, std::string* why) {
   if (c->d_model % 8 || c->d_ffn % 8 || (c->n_heads * c->head_dim) % 8) { *why = "widths must be multiples of 8"; return false; }
   if (c->n_medusa < 0 || c->n_medusa > SPEC_MAX_HEADS) { *why = "n_medusa out of range"; return false; }
   if (c->accept_mode != 0 && c->accept_mode != 1) { *why = "accept_mode must be 0 or 1"; return false; }
+  if (c->sampling != 0 && c->sampling != 1) { *why = "sampling must be 0 or 1"; return false; }
+  if (c->sampling && (c->accept_mode != 1 || !(c->temperature > 0.f))) { *why = "sampled decoding needs accept_mode 1 and a positive temperature"; return false; }
   bool tc = c->dtype == 1 && !(c->flags & SPEC_FLAG_SIMPLE_KERNELS);
   if ((c->flags & SPEC_FLAG_PACKED_WEIGHTS) && !tc) { *why = "pre-tiled weights need the bf16 tensor-core path"; return false; }
   if (tc) {
@@ -331,6 +349,7 @@ size_t carve(spec_ctx* c, void* base) {
   c->d_trace = b.take<unsigned long long>((size_t)TRACE_CAP * 4);
   c->d_attn_arrive = b.take<unsigned int>((size_t)B * f.n_heads);
   c->d_pval2 = b.take<float>(c->Mcap); c->d_pidx2 = b.take<int>(c->Mcap);
+  c->d_draws = b.take<int>(B);
   c->d_n = b.take<int>(B); c->d_cnt = b.take<int>(B); c->d_n_old = b.take<int>(B); c->d_root = b.take<int>(B);
   c->d_count = b.take<int>(B); c->d_path = b.take<int>((size_t)B * (K + 1)); c->d_out_tok = b.take<int>((size_t)B * (K + 1));
   c->d_gen_cnt = b.take<int>(B); c->d_gen_log = b.take<int>((size_t)B * c->gen_cap);
@@ -458,6 +477,47 @@ int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* c
   GemmPlan g;
   int tiles_all = 0;
   for (int i = 0; i < n_mats; ++i) tiles_all += (rows[i] + 127) / 128;
+  if (M > 128 && c->wide_gemm && K % 64 == 0 && n_mats <= GS_MAX_MATS) {
+    // many rows: the compute-bound kernel, whole tiles (one "slot" of finished sums)
+    WideGemmParams w{};
+    w.M = M; w.K = K; w.KC = K / 64; w.n_mats = n_mats;
+    int t0 = 0;
+    StreamTmaps tmw{};
+    for (int i = 0; i < n_mats; ++i) {
+      w.mat_tile0[i] = t0;
+      t0 += (rows[i] + 127) / 128;
+      if (c->packed) { w.packed[i] = static_cast<const uint8_t*>(mats[i]); continue; }
+      const CUtensorMap* t = c->tmap(mats[i], rows[i], K, 128);
+      if (!t) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed (weights)");
+      tmw.a[i] = *t;
+    }
+    for (int i = n_mats; i <= GS_MAX_MATS; ++i) w.mat_tile0[i] = t0;
+    w.n_tiles = tiles_all; w.m_tiles = (M + GW_NT - 1) / GW_NT;
+    const long long total = (long long)w.n_tiles * w.m_tiles * w.KC;
+    if ((size_t)M * tiles_all * 128 > c->part_floats) return c->fail(SPEC_E_NOMEM, "partial-sum scratch too small");
+    if (total > 0x3fffffff || (total + 1) * (long long)(w.n_tiles * w.m_tiles) >= 0x7fffffffLL) return c->fail(SPEC_E_BADARG, "unsupported linear shape");
+    const CUtensorMap* tb = c->tmap(x, std::max<size_t>(round_up(M, 16), GW_NT), K, GW_NT);
+    if (!tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed (activations)");
+    tmw.b = *tb;
+    w.part = c->d_part; w.status = c->d_status; w.trace = c->next_trace(gemm_kind_name(kind));
+    const int grid = std::min(w.n_tiles * w.m_tiles, SM_SLOTS / 2);
+    {
+      ProfScope ps(c, kind);
+      static bool set_dev[kAttrDevices] = {};
+      bool& set_ = *attr_flag(set_dev);
+      if (!set_) { CUDA_OK(cudaFuncSetAttribute(gemm_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, WideCfg::SMEM_BYTES)); set_ = true; }
+      cudaError_t e = launch_k(c->pdl, gemm_wide, dim3(grid), dim3(192), (size_t)WideCfg::SMEM_BYTES, c->stream, tmw, w);
+      c->launches++;
+      if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_wide launch: ") + cudaGetErrorString(e));
+    }
+    // the consumers see one finished slot per tile: a dealing of the units with one CTA per (weight tile, 256-row tile)
+    PartView v{};
+    v.part = c->d_part; v.slot_stride = (size_t)M * tiles_all * 128; v.ld = tiles_all * 128;
+    v.seg.KC = w.KC; v.seg.m_tiles = w.m_tiles; v.seg.G = w.n_tiles * w.m_tiles; v.seg.total = (int)total;
+    v.mt_shift = 8;
+    *view = v;
+    return SPEC_OK;
+  }
   const int g_cap = aligned_ctas(tiles_all, tiles_all <= 48 ? std::min(c->gemm_ctas, c->small_gemm_ctas) : c->gemm_ctas);
   if (!plan_gemm(M, K, n_mats, rows, g_cap, &g))
     return c->fail(SPEC_E_BADARG, "unsupported linear shape");
@@ -484,6 +544,100 @@ int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* c
     if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_stream launch: ") + cudaGetErrorString(e));
   }
   *view = plan_view(g);
+  return SPEC_OK;
+}
+
+// Can the cluster-reduced GEMM take this shape? One activation tile, and enough K chunks for every CTA
+// of the cluster to get a run (GC_SWIGLU also needs both accumulators of the middle CTA staged at once).
+bool cluster_gemm_ok(const spec_ctx* c, int mode, int M, int K) {
+  const int bit = mode == GC_RESIDUAL ? 1 : (mode == GC_SWIGLU ? 2 : 4);
+  if (!(c->cluster_epilogue & bit) || M < 1 || M > 128 || K % 64) return false;
+  const int KC = K / 64;
+  if (mode == GC_RESIDUAL) return KC >= GC_RES_CLUSTER;
+  if (mode == GC_SWIGLU) return KC >= 3 && M <= 64;
+  return KC >= GC_ROPE_CLUSTER && (c->cfg.head_dim == 64 || c->cfg.head_dim == 128);
+}
+
+template <int MT, int MODE>
+cudaError_t launch_gc_mt(cudaStream_t st, bool pdl, int grid, const StreamTmaps& tm, const ClusterGemmParams& p, bool* attr_set) {
+  if (!*attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_cluster<MT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, ClusterCfg<MT>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    *attr_set = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = (size_t)ClusterCfg<MT>::SMEM_BYTES; cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = MODE == GC_RESIDUAL ? GC_RES_CLUSTER : (MODE == GC_SWIGLU ? GC_GLU_CLUSTER : GC_ROPE_CLUSTER);
+  at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, gemm_cluster<MT, MODE>, tm, p);
+}
+
+// x[M,N] += in[M,K] * W^T (GC_RESIDUAL, mats[0] = W), act_out[M,N] = bf16(SiLU(in W_g^T) * in W_u^T)
+// (GC_SWIGLU, mats = gate, up) or q / cache rows of layer `layer` = RoPE(in [W_q; W_k; W_v]^T) (GC_ROPE, mats =
+// q, k, v; rows = the pass's row bookkeeping), finished inside the kernel. Caller checked cluster_gemm_ok.
+int run_gemm_cluster(spec_ctx* c, int mode, const void* in, int M, int K, const void* const* mats, int N, float* x,
+                     bf16* act_out, int kind, int layer = -1, const Rows* rows = nullptr) {
+  const spec_config& f = c->cfg;
+  const int MT = mt_for_rows(M), n_mats = mode == GC_RESIDUAL ? 1 : (mode == GC_SWIGLU ? 2 : 3);
+  ClusterGemmParams p{};
+  p.M = M; p.K = K; p.KC = K / 64; p.N = N;
+  const int HD = f.n_heads * f.head_dim, KD = f.n_kv_heads * f.head_dim;
+  StreamTmaps tm{};
+  for (int i = 0; i < n_mats; ++i) {
+    if (c->packed) { p.packed[i] = static_cast<const uint8_t*>(mats[i]); continue; }
+    const int rws = mode == GC_ROPE ? (i == 0 ? HD : KD) : N;
+    const CUtensorMap* t = c->tmap(mats[i], rws, K, 128);
+    if (!t) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed (weights)");
+    tm.a[i] = *t;
+  }
+  const CUtensorMap* tb = c->tmap(in, std::max<size_t>(round_up(M, 16), MT), K, MT);
+  if (!tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed (activations)");
+  tm.b = *tb;
+  p.x = x; p.ss_part = nullptr; p.act = act_out; p.status = c->d_status;
+  int n_tiles = (N + 127) / 128;
+  if (mode == GC_ROPE) {
+    const int tq = (HD + 127) / 128, tk = (KD + 127) / 128;
+    p.tile0[0] = 0; p.tile0[1] = tq; p.tile0[2] = tq + tk;
+    n_tiles = tq + 2 * tk;
+    p.H = f.n_heads; p.layer = layer; p.rows = *rows; p.cs = c->d_rope; p.q = static_cast<bf16*>(c->d_q);
+    p.pool = static_cast<bf16*>(c->d_pool); p.g = c->geom; p.page_table = c->d_page_table;
+  }
+  p.trace = c->next_trace(gemm_kind_name(kind));
+  const int grid = n_tiles * (mode == GC_RESIDUAL ? GC_RES_CLUSTER : (mode == GC_SWIGLU ? GC_GLU_CLUSTER : GC_ROPE_CLUSTER));
+  cudaError_t e = cudaErrorInvalidValue;
+  {
+    ProfScope ps(c, kind);
+    bool* as = c->gc_attr_set;
+    if (mode == GC_RESIDUAL) {
+      switch (MT) {
+        case 16: e = launch_gc_mt<16, GC_RESIDUAL>(c->stream, c->pdl, grid, tm, p, as + 0); break;
+        case 32: e = launch_gc_mt<32, GC_RESIDUAL>(c->stream, c->pdl, grid, tm, p, as + 1); break;
+        case 64: e = launch_gc_mt<64, GC_RESIDUAL>(c->stream, c->pdl, grid, tm, p, as + 2); break;
+        default: e = launch_gc_mt<128, GC_RESIDUAL>(c->stream, c->pdl, grid, tm, p, as + 3); break;
+      }
+    } else if (mode == GC_SWIGLU) {
+      switch (MT) {
+        case 16: e = launch_gc_mt<16, GC_SWIGLU>(c->stream, c->pdl, grid, tm, p, as + 4); break;
+        case 32: e = launch_gc_mt<32, GC_SWIGLU>(c->stream, c->pdl, grid, tm, p, as + 5); break;
+        default: e = launch_gc_mt<64, GC_SWIGLU>(c->stream, c->pdl, grid, tm, p, as + 6); break;
+      }
+    } else {
+      switch (MT) {
+        case 16: e = launch_gc_mt<16, GC_ROPE>(c->stream, c->pdl, grid, tm, p, as + 7); break;
+        case 32: e = launch_gc_mt<32, GC_ROPE>(c->stream, c->pdl, grid, tm, p, as + 8); break;
+        case 64: e = launch_gc_mt<64, GC_ROPE>(c->stream, c->pdl, grid, tm, p, as + 9); break;
+        default: e = launch_gc_mt<128, GC_ROPE>(c->stream, c->pdl, grid, tm, p, as + 10); break;
+      }
+    }
+    c->launches++;
+  }
+  if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_cluster launch: ") + cudaGetErrorString(e));
   return SPEC_OK;
 }
 
@@ -533,11 +687,13 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
     dim3 grid(H, nw, c->B);
     ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
     if (D == 128) {
-      static bool set_ = false;
+      static bool set_dev[kAttrDevices] = {};
+      bool& set_ = *attr_flag(set_dev);
       if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_rows<128, ATTN_ROWS_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_rows_smem(128, ATTN_ROWS_WARPS))); set_ = true; }
       KLAUNCH("attention_tc", (attention_rows<128, ATTN_ROWS_WARPS>), grid, dim3(ATTN_ROWS_WARPS * 32), attention_rows_smem(128, ATTN_ROWS_WARPS), a);
     } else {
-      static bool set_ = false;
+      static bool set_dev[kAttrDevices] = {};
+      bool& set_ = *attr_flag(set_dev);
       if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_rows<64, ATTN_ROWS_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_rows_smem(64, ATTN_ROWS_WARPS))); set_ = true; }
       KLAUNCH("attention_tc", (attention_rows<64, ATTN_ROWS_WARPS>), grid, dim3(ATTN_ROWS_WARPS * 32), attention_rows_smem(64, ATTN_ROWS_WARPS), a);
     }
@@ -554,7 +710,8 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
 #define ATTN_CASE(HDV, NWV, KGV)                                                                         \
   {                                                                                                    \
     size_t sm = attention_tc_smem(HDV, NWV, a.stages);                                                 \
-    static bool set_ = false;                                                                          \
+    static bool set_dev[kAttrDevices] = {};                                                            \
+    bool& set_ = *attr_flag(set_dev);                                                                  \
     if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_tc<HDV, NWV, KGV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_tc_smem(HDV, NWV, ATTN_MAX_STAGES))); set_ = true; } \
     KLAUNCH("attention_tc", (attention_tc<HDV, NWV, KGV>), grid, dim3(NWV * KGV * 32), sm, a);         \
   }
@@ -588,37 +745,50 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, cons
   for (int l = 0; l < f.n_layers; ++l) {
     NORM_LAUNCH(pend, c->an[l], u, (float*)nullptr);
     int r;
-    PartView vq{};
     {
       const void* mats[3] = {c->wq[l], c->wk[l], c->wv[l]};
       int rws[3] = {HD, KD, KD};
-      if ((r = run_gemm(c, u, M, d, 3, mats, rws, SPEC_PROFILE_QKV, &vq))) return r;
+      if (cluster_gemm_ok(c, GC_ROPE, M, d)) {
+        // the clusters rotate q and k and store q and the cache rows themselves
+        if ((r = run_gemm_cluster(c, GC_ROPE, u, M, d, mats, 0, nullptr, nullptr, SPEC_PROFILE_QKV, l, &rows))) return r;
+      } else {
+        PartView vq{};
+        if ((r = run_gemm(c, u, M, d, 3, mats, rws, SPEC_PROFILE_QKV, &vq))) return r;
+        KLAUNCH("rope_store_tc", rope_store_tc, dim3(M, M <= 128 ? 8 : 1), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope,
+                static_cast<bf16*>(c->d_q), static_cast<bf16*>(c->d_pool), c->geom, c->d_page_table, l, H);
+      }
     }
-    KLAUNCH("rope_store_tc", rope_store_tc, dim3(M, M <= 128 ? 8 : 1), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope,
-            static_cast<bf16*>(c->d_q), static_cast<bf16*>(c->d_pool), c->geom, c->d_page_table, l, H);
     if ((r = launch_attention_tc(c, rows, R, l, n_hi_pass, n_lo_pass))) return r;
     PartView vo{};
     {
       const void* mats[1] = {c->wo[l]};
       int rws[1] = {d};
-      if ((r = run_gemm(c, c->d_attn, M, HD, 1, mats, rws, SPEC_PROFILE_WO, &vo))) return r;
+      if (cluster_gemm_ok(c, GC_RESIDUAL, M, HD)) {
+        // the cluster adds its split-K sums and the residual stream itself: nothing left for the norm kernel to add
+        if ((r = run_gemm_cluster(c, GC_RESIDUAL, c->d_attn, M, HD, mats, d, c->d_x, nullptr, SPEC_PROFILE_WO))) return r;
+      } else if ((r = run_gemm(c, c->d_attn, M, HD, 1, mats, rws, SPEC_PROFILE_WO, &vo))) return r;
     }
     NORM_LAUNCH(vo, c->fn[l], u, (float*)nullptr);
-    PartView vg{};
     {
       const void* mats[2] = {c->wg[l], c->wu[l]};
       int rws[2] = {F, F};
-      if ((r = run_gemm(c, u, M, d, 2, mats, rws, SPEC_PROFILE_GATE_UP, &vg))) return r;
-    }
-    {
-      size_t total = (size_t)M * (F / 4);
-      unsigned blocks = (unsigned)std::min<size_t>((total + 255) / 256, 2 * SM_SLOTS);
-      KLAUNCH("swiglu_reduce_tc", swiglu_reduce_tc, dim3(blocks), dim3(256), 0, vg, 0, up0, act, M, F);
+      if (cluster_gemm_ok(c, GC_SWIGLU, M, d)) {
+        if ((r = run_gemm_cluster(c, GC_SWIGLU, u, M, d, mats, F, nullptr, act, SPEC_PROFILE_GATE_UP))) return r;
+      } else {
+        PartView vg{};
+        if ((r = run_gemm(c, u, M, d, 2, mats, rws, SPEC_PROFILE_GATE_UP, &vg))) return r;
+        size_t total = (size_t)M * (F / 4);
+        unsigned blocks = (unsigned)std::min<size_t>((total + 255) / 256, 2 * SM_SLOTS);
+        KLAUNCH("swiglu_reduce_tc", swiglu_reduce_tc, dim3(blocks), dim3(256), 0, vg, 0, up0, act, M, F);
+      }
     }
     {
       const void* mats[1] = {c->wd[l]};
       int rws[1] = {d};
-      if ((r = run_gemm(c, act, M, F, 1, mats, rws, SPEC_PROFILE_DOWN, &pend))) return r;
+      pend = PartView{};
+      if (cluster_gemm_ok(c, GC_RESIDUAL, M, F)) {
+        if ((r = run_gemm_cluster(c, GC_RESIDUAL, act, M, F, mats, d, c->d_x, nullptr, SPEC_PROFILE_DOWN))) return r;
+      } else if ((r = run_gemm(c, act, M, F, 1, mats, rws, SPEC_PROFILE_DOWN, &pend))) return r;
     }
   }
   NORM_LAUNCH(pend, c->final_norm, static_cast<bf16*>(c->d_hq), c->d_hid);
@@ -776,6 +946,7 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
   CUDA_OK(cudaMemcpyAsync(c->d_prompt, tokens + offsets[0], (size_t)off[batch] * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CUDA_OK(cudaMemcpyAsync(c->d_offsets, off.data(), (batch + 1) * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CUDA_OK(cudaMemsetAsync(c->d_gen_cnt, 0, batch * sizeof(int), c->stream));
+  CUDA_OK(cudaMemsetAsync(c->d_draws, 0, batch * sizeof(int), c->stream));
   CUDA_OK(cudaStreamSynchronize(c->stream));   // host staging vector goes out of scope below
   int R = PREFILL_ROWS, M = batch * R;
   Rows rows = make_rows(c, R, true);
@@ -795,6 +966,11 @@ int prefill_t(spec_ctx* c, int batch, const int32_t* tokens, const int32_t* offs
   if (r) return r;
   AcceptArgs a = make_accept(c, 1, 1);
   KLAUNCH("accept_kernel", accept_kernel, dim3(batch), dim3(256), 0, a);
+  if (f.sampling) {
+    sample_root<<<batch, 256, 0, c->stream>>>(c->d_logits, f.vocab, 1, c->K, c->d_path, c->d_count, f.temperature, f.seed_lo,
+                                              f.seed_hi, c->d_draws, c->d_root, 1);
+    LAUNCH_CHECK("sample_root");
+  }
   r = check_status(c);
   if (r) return r;
   c->n_hi.assign(batch, 0);
@@ -863,6 +1039,11 @@ int step_body(spec_ctx* c, const int* ov, const int* n_hi_plan, const int* n_lo_
     a.edge_ok = c->d_edge;
   }
   KLAUNCH("accept_kernel", accept_kernel, dim3(B), dim3(256), 0, a);
+  if (f.sampling) {
+    sample_root<<<B, 256, 0, c->stream>>>(c->d_logits, f.vocab, T_, K, c->d_path, c->d_count, f.temperature, f.seed_lo,
+                                          f.seed_hi, c->d_draws, c->d_root, 0);
+    LAUNCH_CHECK("sample_root");
+  }
   step_event(c, 4);
   // (5) KV compaction
   dim3 gc(f.n_layers * 2 * f.n_kv_heads, B);
@@ -1146,6 +1327,7 @@ int64_t spec_query(const spec_ctx* c, int32_t what) {
     case SPEC_Q_N_NODES: return c->T;
     case SPEC_Q_BATCH: return c->B;
     case SPEC_Q_GRAPH_CAPTURES: return c->graph_captures;
+    case SPEC_Q_CLUSTER_GATE_UP: return c->tc && cluster_gemm_ok(c, GC_SWIGLU, c->B * c->T, f.d_model) ? 1 : 0;
     case SPEC_Q_ALGO_BYTES_PER_STEP: {
       double d = f.d_model, F = f.d_ffn, V = f.vocab, HD = (double)f.n_heads * f.head_dim, KD = (double)f.n_kv_heads * f.head_dim;
       double layer = d * HD + 2 * d * KD + HD * d + 3 * d * F;
@@ -1158,7 +1340,17 @@ int64_t spec_query(const spec_ctx* c, int32_t what) {
 
 int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
   if (!c) return SPEC_E_BADARG;
-  c->graph_epoch++;   // a recorded step no longer matches the options
+  switch (what) {
+    case SPEC_OPT_GEMM_CTAS: case SPEC_OPT_SMALL_GEMM_CTAS:
+      if (value < 1 || value > SM_SLOTS) return c->fail(SPEC_E_BADARG, "gemm CTA count out of range");
+      break;
+    case SPEC_OPT_L2_PREFETCH:
+      if (value < 0 || value > 64) return c->fail(SPEC_E_BADARG, "L2 prefetch depth out of range");
+      break;
+    case SPEC_OPT_GRAPH: case SPEC_OPT_PHASE_TIMING: case SPEC_OPT_PDL: case SPEC_OPT_TRACE: case SPEC_OPT_CLUSTER_EPILOGUE: case SPEC_OPT_WIDE_GEMM: break;
+    default: return c->fail(SPEC_E_BADARG, "unknown option");
+  }
+  c->graph_epoch++;   // the option is valid: a recorded step no longer matches the options
   switch (what) {
     case SPEC_OPT_GRAPH:
       c->graph_on = value != 0; return SPEC_OK;
@@ -1174,6 +1366,8 @@ int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
     case SPEC_OPT_SMALL_GEMM_CTAS:
       if (value < 1 || value > SM_SLOTS) return c->fail(SPEC_E_BADARG, "out of range");
       c->small_gemm_ctas = value; return SPEC_OK;
+    case SPEC_OPT_CLUSTER_EPILOGUE: c->cluster_epilogue = value & 7; return SPEC_OK;
+    case SPEC_OPT_WIDE_GEMM: c->wide_gemm = value != 0; return SPEC_OK;
     case SPEC_OPT_TRACE:
       c->trace_on = value != 0;
       if (c->trace_on && c->trace_init.empty()) {
@@ -1249,6 +1443,19 @@ int spec_debug_read(spec_ctx* c, int32_t what, void* host_buf, size_t bytes) {
   CUDA_OK(cudaMemcpyAsync(host_buf, src, need, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(cudaStreamSynchronize(c->stream));
   return SPEC_OK;
+}
+
+int spec_debug_wait_timeout(spec_ctx* c, int32_t limit_us) {
+  if (!c) return SPEC_E_BADARG;
+  if (limit_us < 1 || limit_us > 100000) return c->fail(SPEC_E_BADARG, "limit must be 1..100000 microseconds");
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  wait_probe<<<1, 32, 0, c->stream>>>(c->d_status, (unsigned long long)limit_us * 1000ull);
+  LAUNCH_CHECK("wait_probe");
+  int r = check_status(c);           // reads the status word: SPEC_E_TIMEOUT with the probe's place code
+  // the probe is the only writer here: clear the word so that the context stays usable
+  CUDA_OK(cudaMemsetAsync(c->d_status, 0, 4 * sizeof(int), c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  return r;
 }
 
 int spec_debug_read_kv(spec_ctx* c, int32_t seq, int32_t layer, int32_t slot0, int32_t n_slots, float* host_k, float* host_v) {

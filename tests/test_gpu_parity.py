@@ -81,6 +81,33 @@ def test_small_bf16_d128_tree64_tensor_core_path(torch):
     assert rep.max_logit_err < TOL_BF16
 
 
+def test_small_bf16_d512_cluster_epilogues(torch):
+    """A width at which every projection with a cluster epilogue takes it (output projection K = 512 = 8
+    chunks for the 8-CTA cluster; gate+up as clusters of 3 with the SwiGLU inside; down projection
+    K = 1344; q/k/v with RoPE and the cache store inside), with a d_ffn that leaves the last tile half empty,
+    against the oracle: all cluster epilogues on, the default set, none, and smaller trees."""
+    from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights
+    from paper_2503_14153_b200 import binding as B
+    from tests_lockstep import run_lockstep
+    cfg = SMALL_BF16.with_(name="small_bf16_d512", d_model=512, n_heads=4, n_kv_heads=4, head_dim=128, d_ffn=1344,
+                           n_medusa=4, topk=(10, 4, 2, 2), tree_nodes=64, seed=24)
+    w, prompt = draw_weights(cfg), draw_prompt(cfg, 150)
+    tree = build_tree(cfg.topk, cfg.tree_nodes)
+    dw = upload_weights(cfg, w)
+    for mask in (7, 2, 0):        # every cluster epilogue; the default (gate+up only); none
+        gpu = SpecDecoder(cfg, dw, tree, 150 + 24 + 8, flags=B.FLAG_KEEP_LOGITS)
+        gpu.set_option(B.OPT_CLUSTER_EPILOGUE, mask)
+        rep = run_lockstep(cfg, w, tree, prompt, 24, TOL_BF16, TIE_GAP, check_kv_every=3, gpu=gpu)
+        gpu.close()
+        assert rep.steps > 0
+    for T in (16, 32):
+        gpu = SpecDecoder(cfg, dw, build_tree(cfg.topk, T), 40 + 8 + 8, flags=B.FLAG_KEEP_LOGITS)
+        gpu.set_option(B.OPT_CLUSTER_EPILOGUE, 7)
+        r2 = run_lockstep(cfg, w, build_tree(cfg.topk, T), prompt[:40], 8, TOL_BF16, TIE_GAP, gpu=gpu)
+        gpu.close()
+        assert r2.steps > 0
+
+
 def test_ten_heads_deep_tree(torch):
     """The paper's head count (K = 10): ten stacked head matrices (three GEMM launches), a tree ten levels deep."""
     cfg = SMALL_BF16.with_(name="small_bf16_k10", n_medusa=10, topk=(4, 3, 2, 2, 2, 1, 1, 1, 1, 1), tree_nodes=48, seed=23)
@@ -134,6 +161,30 @@ def test_typical_acceptance_mode(torch):
     cfg = get_config("c0")
     rep = _lockstep(cfg, TOL_FP32, 30, accept_mode=1, typ=(0.3, 0.6, 1.0))
     assert rep.steps > 0
+
+
+@pytest.mark.parametrize("temperature", [0.5, 2.0])
+def test_typical_acceptance_at_a_temperature(torch, temperature):
+    """Eq. 1 with p = softmax(logits / temperature), temperature != 1, argmax next token."""
+    cfg = get_config("c0")
+    rep = _lockstep(cfg, TOL_FP32, 30, accept_mode=1, typ=(0.3, 0.6, temperature))
+    assert rep.steps > 0 and max(rep.counts) > 1
+
+
+@pytest.mark.parametrize("seed", [7, (5 << 32) + 11])
+def test_sampled_decoding_temperature_0p8(torch, seed):
+    """Sampled decoding at temperature 0.8 (Sec. IV-B times every prompt greedy and sampled): Eq. 1
+    acceptance and the next token drawn at the step's Philox uniform, token for token against the
+    oracle (both sides draw the same uniforms; a draw may differ only at a boundary of the
+    cumulative distribution)."""
+    cfg = get_config("c0")
+    t = float(np.float32(0.8))          # the value the float32 field of the configuration holds
+    rep = _lockstep(cfg, TOL_FP32, 48, accept_mode=1, typ=(0.09, 0.3, t), sampling=True, seed=seed)
+    assert rep.steps > 0 and len(rep.near_ties) <= 1
+    greedy = _lockstep(cfg, TOL_FP32, 48, accept_mode=1, typ=(0.09, 0.3, t))
+    assert rep.tokens != greedy.tokens          # the draws matter: not the argmax stream
+    other = _lockstep(cfg, TOL_FP32, 16, accept_mode=1, typ=(0.09, 0.3, t), sampling=True, seed=seed + 1)
+    assert other.tokens[:16] != rep.tokens[:16]
 
 
 @pytest.mark.parametrize("M,N,K,ctas", [(16, 128, 64, 1), (64, 384, 256, 2), (64, 4096, 4096, 296),
@@ -210,6 +261,32 @@ def test_error_returns_and_degenerate_shapes(torch):
         tok, cnt = dec.step()
         assert int(cnt[0]) == 1
     dec.close()
+
+
+def test_bounded_wait_times_out_and_context_survives(torch):
+    """A device-side wait that nothing completes gives up after its limit: the library reports
+    SPEC_E_TIMEOUT with the place code, and the same context decodes on afterwards."""
+    from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights
+    cfg = get_config("c0")
+    w = draw_weights(cfg)
+    dec = SpecDecoder(cfg, upload_weights(cfg, w), build_tree(cfg.topk, cfg.tree_nodes), max_seq=96)
+    prompt = draw_prompt(cfg)
+    dec.prefill(prompt)
+    tok0, cnt0 = dec.step()
+    assert dec.wait_timeout_probe(1000) == -6                 # SPEC_E_TIMEOUT after 1 ms
+    msg = dec.lib.spec_last_error(dec._ctx).decode()
+    assert "status 1 at 99" in msg, msg
+    assert dec.wait_timeout_probe(0) == -1                    # limit out of range: refused, nothing launched
+    assert dec.debug(5 + 5)[0] == 0                           # status word is clean again (SPEC_DBG_STATUS)
+    tok1, cnt1 = dec.step()                                   # the context is still usable
+    assert 1 <= int(cnt1[0]) <= cfg.n_medusa + 1
+    # and the stream is what an undisturbed decoder emits
+    ref = SpecDecoder(cfg, upload_weights(cfg, w), build_tree(cfg.topk, cfg.tree_nodes), max_seq=96)
+    ref.prefill(prompt)
+    a, ca = ref.step()
+    b, cb = ref.step()
+    assert list(a[0][:int(ca[0])]) == list(tok0[0][:int(cnt0[0])]) and list(b[0][:int(cb[0])]) == list(tok1[0][:int(cnt1[0])])
+    dec.close(); ref.close()
 
 
 def test_timeline_and_options(torch):

@@ -42,8 +42,14 @@ def test_static_scratch_linear_matches_caller_scratch_linear_twice(torch):
         want = spec_op_linear(x, w, ctas)
         y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")   # caller-owned output
         before = torch.cuda.memory_stats()["allocation.all.allocated"]    # cumulative count of allocations
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]                        # what the driver says is free on the device
         got = spec_op_linear_static(x, w, y, ctas)
         assert torch.cuda.memory_stats()["allocation.all.allocated"] == before   # none came from torch's allocator
+        if (M, N, K) != cases[0][:3]:
+            # (the library links the CUDA runtime statically, so an allocation of its own would not show in torch's
+            # counters: after the first call, which may load the kernels' code, the device's free memory must not move)
+            assert torch.cuda.mem_get_info()[0] == free_before
         torch.cuda.synchronize()
         err = (got - want).abs().max().item() / want.abs().max().item()
         assert err <= TOL, (M, N, K, ctas, err)
