@@ -223,6 +223,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, per-kernel and CPU legs (profiling)")
     ap.add_argument("--cluster-epilogues", type=int, default=None, help="SPEC_OPT_CLUSTER_EPILOGUE bit mask (A/B measurements)")
     ap.add_argument("--wide-gemm", type=int, default=None, help="SPEC_OPT_WIDE_GEMM (A/B measurements of the batched configuration)")
+    ap.add_argument("--long-attn-keys", type=int, default=None, help="SPEC_OPT_LONG_ATTN_KEYS (A/B measurements)")
+    ap.add_argument("--attn-umma", type=int, default=None, help="SPEC_OPT_ATTN_UMMA (A/B measurements)")
     ap.add_argument("--reference-budget-s", type=float, default=150.0, help="wall budget of the reference arm's timed steps")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -270,6 +272,10 @@ def main():
         dec.set_option(B.OPT_CLUSTER_EPILOGUE, args.cluster_epilogues)
     if args.wide_gemm is not None:
         dec.set_option(B.OPT_WIDE_GEMM, args.wide_gemm)
+    if args.attn_umma is not None:
+        dec.set_option(B.OPT_ATTN_UMMA, args.attn_umma)
+    if args.long_attn_keys is not None:
+        dec.set_option(B.OPT_LONG_ATTN_KEYS, args.long_attn_keys)
     peak, peak_kind = measured_peaks()
 
     def barrier():

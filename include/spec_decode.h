@@ -156,7 +156,8 @@ const char *spec_last_error(const spec_ctx *ctx);
 enum { SPEC_Q_KMAX = 0, SPEC_Q_KERNEL_LAUNCHES = 1, SPEC_Q_N_NODES = 2, SPEC_Q_BATCH = 3,
        SPEC_Q_ALGO_BYTES_PER_STEP = 4 /* weights + lm_head (twice) + heads, in KiB */,
        SPEC_Q_GRAPH_CAPTURES = 5 /* times a step was recorded into a CUDA graph */,
-       SPEC_Q_CLUSTER_GATE_UP = 6 /* 1 if a step's gate+up projection runs as the cluster kernel with the SwiGLU inside */ };
+       SPEC_Q_CLUSTER_GATE_UP = 6 /* 1 if a step's gate+up projection runs as the cluster kernel with the SwiGLU inside */,
+       SPEC_Q_WIDE_GEMM = 7 /* 1 if passes of more than 128 rows use the 128 x 256-tile kernel */ };
 int64_t spec_query(const spec_ctx *ctx, int32_t what);
 
 /* Tuning knobs of a context (defaults in brackets). SPEC_OPT_PDL [1]: launch the kernels of
@@ -184,10 +185,14 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
  * faster (bits 1 and 4 cost 2% and 4% of a step there). SPEC_OPT_WIDE_GEMM [1]: passes of more than
  * 128 rows (batched verification, batched prompt processing) run their projections as whole
  * [128 weight rows] x [256 activation rows] tiles that keep a weight tile for 256 rows at a time;
- * 0 = the weight-streaming kernel, which re-reads the weights for every 128 rows. */
+ * 0 = the weight-streaming kernel, which re-reads the weights for every 128 rows.
+ * SPEC_OPT_LONG_ATTN_KEYS [2048]: passes of more than 32 rows whose context may exceed this many positions
+ * run the attention kernel that shares each K/V tile among the row blocks of a CTA and splits the keys
+ * across CTAs (0 = never). Results differ from the other attention kernels only in summation order. */
 enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2, SPEC_OPT_TRACE = 3,
        SPEC_OPT_SMALL_GEMM_CTAS = 4, SPEC_OPT_GRAPH = 5, SPEC_OPT_PHASE_TIMING = 6, SPEC_OPT_CLUSTER_EPILOGUE = 7,
-       SPEC_OPT_WIDE_GEMM = 8 };
+       SPEC_OPT_WIDE_GEMM = 8, SPEC_OPT_LONG_ATTN_KEYS = 9,
+       SPEC_OPT_ATTN_UMMA = 10 };
 int spec_set_option(spec_ctx *ctx, int32_t what, int32_t value);
 
 /* Device timeline of the LAST step, recorded while SPEC_OPT_TRACE is on: one record per kernel

@@ -19,8 +19,8 @@ FLAG_SIMPLE_KERNELS = 2
 FLAG_PACKED_WEIGHTS = 4
 PROFILE_OFF, PROFILE_GATE_UP, PROFILE_QKV, PROFILE_WO, PROFILE_DOWN, PROFILE_ATTENTION = range(6)
 
-Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB, Q_GRAPH_CAPTURES, Q_CLUSTER_GATE_UP = 0, 1, 2, 3, 4, 5, 6
-OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH, OPT_TRACE, OPT_SMALL_GEMM_CTAS, OPT_GRAPH, OPT_PHASE_TIMING, OPT_CLUSTER_EPILOGUE, OPT_WIDE_GEMM = 0, 1, 2, 3, 4, 5, 6, 7, 8
+Q_KMAX, Q_KERNEL_LAUNCHES, Q_N_NODES, Q_BATCH, Q_ALGO_KIB, Q_GRAPH_CAPTURES, Q_CLUSTER_GATE_UP, Q_WIDE_GEMM = 0, 1, 2, 3, 4, 5, 6, 7
+OPT_PDL, OPT_GEMM_CTAS, OPT_L2_PREFETCH, OPT_TRACE, OPT_SMALL_GEMM_CTAS, OPT_GRAPH, OPT_PHASE_TIMING, OPT_CLUSTER_EPILOGUE, OPT_WIDE_GEMM, OPT_LONG_ATTN_KEYS, OPT_ATTN_UMMA = 0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10
 TRACE_NAME_LEN = 32
 (DBG_TOK, DBG_POS, DBG_LOGITS, DBG_HIDDEN, DBG_ARGMAX, DBG_PATH, DBG_CAND, DBG_SEQLEN, DBG_NEXT_ROOT,
  DBG_H_LAST, DBG_STATUS) = range(11)
@@ -358,8 +358,11 @@ class SpecDecoder:
 
     def gate_up_kernel_name(self) -> str:
         """Name of the kernel a step's gate+up projection runs as (the dominant kernel of a 7B step)."""
-        mt = 16 if self.batch * self.T <= 16 else (32 if self.batch * self.T <= 32 else (64 if self.batch * self.T <= 64 else 128))
-        return f"gemm_cluster<{mt},swiglu>" if self.query(Q_CLUSTER_GATE_UP) else f"gemm_stream<{mt}>"
+        m = self.batch * self.T
+        mt = 16 if m <= 16 else (32 if m <= 32 else (64 if m <= 64 else 128))
+        if self.query(Q_CLUSTER_GATE_UP):
+            return f"gemm_cluster<{mt},swiglu>"
+        return "gemm_wide" if m > 128 and self.query(Q_WIDE_GEMM) else f"gemm_stream<{mt}>"
 
     def query(self, what: int) -> int:
         return int(self.lib.spec_query(self._ctx, what))

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspec_decode.so")
 SOURCES = ["spec_api.cu"]
-DEPS = ["spec_api.cu", "common.cuh", "kernels_simple.cuh", "gemm_stream.cuh", "gemm_cluster.cuh", "gemm_wide.cuh", "glue_tc.cuh", "attention_tc.cuh", "labels.cuh",
+DEPS = ["spec_api.cu", "common.cuh", "kernels_simple.cuh", "gemm_stream.cuh", "gemm_cluster.cuh", "gemm_wide.cuh", "glue_tc.cuh", "attention_tc.cuh", "attention_umma.cuh", "labels.cuh",
         os.path.join("..", "..", "include", "spec_decode.h")]
 
 

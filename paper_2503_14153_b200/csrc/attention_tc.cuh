@@ -4,8 +4,8 @@
 // (rg, kg) owns query rows [16 rg, 16 rg + 16) and every KG-th tile of the split, so two
 // tiles are worked on at a time; the key groups' softmax states are merged through shared
 // memory at the end. KV tiles of 64 keys are brought in page by page with bulk asynchronous
-// copies that complete on an mbarrier (the cache's in-page chunk swizzle makes the landed
-// tile conflict-free for ldmatrix); QK^T and PV run on mma.sync m16n8k16 with a warp-level
+// copies that complete on an mbarrier (the cache's slab layout -- 64 dims per 128-byte row, chunks
+// swizzled with the row -- makes the landed tile conflict-free for ldmatrix); QK^T and PV run on mma.sync m16n8k16 with a warp-level
 // online softmax; the tree mask is a 128-bit ancestor set per row applied only to keys at or
 // beyond the committed length. Two kernels: attention_rows (at the end of this file) when the
 // (sequence, head, 16-row block) CTAs of the pass fit the SMs, attention_tc otherwise. For
@@ -229,7 +229,7 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
           for (int j2 = 0; j2 < KT / 16; ++j2) {
             int key = j2 * 16 + (lane & 7) + (lane >> 4) * 8;
             int ch = kk * 2 + ((lane >> 3) & 1);
-            ldmatrix_x4(smem_u32(kt + (key >> 4) * 2 * PAGE_BYTES + (key & 15) * ROWB + ((ch ^ (key & 7)) << 4)), dst[j2]);
+            ldmatrix_x4(smem_u32(kt + (key >> 4) * 2 * PAGE_BYTES + (ch >> 3) * 2048 + (key & 15) * 128 + (((ch & 7) ^ (key & 7)) << 4)), dst[j2]);
           }
         };
         load_k(0, kf[0]);
@@ -294,7 +294,7 @@ attention_tc(const AttnTcArgs a, unsigned long long* tr) {
           for (int dd = 0; dd < DG; ++dd) {
             int key = j * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
             int ch = (d0 + dd) * 2 + (lane >> 4);
-            ldmatrix_x4_trans(smem_u32(vt + (key >> 4) * 2 * PAGE_BYTES + (key & 15) * ROWB + ((ch ^ (key & 7)) << 4)), dst[dd]);
+            ldmatrix_x4_trans(smem_u32(vt + (key >> 4) * 2 * PAGE_BYTES + (ch >> 3) * 2048 + (key & 15) * 128 + (((ch & 7) ^ (key & 7)) << 4)), dst[dd]);
           }
         };
         load_v(0, vf[0]);
@@ -590,7 +590,7 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
         for (int j2 = 0; j2 < SK / 16; ++j2) {
           const int key = j2 * 16 + (lane & 7) + (lane >> 4) * 8;
           const int ch = kk * 2 + ((lane >> 3) & 1);
-          ldmatrix_x4(smem_u32(kt + (key >> 4) * 2 * PAGE_BYTES + (key & 15) * ROWB + ((ch ^ (key & 7)) << 4)), dst[j2]);
+          ldmatrix_x4(smem_u32(kt + (key >> 4) * 2 * PAGE_BYTES + (ch >> 3) * 2048 + (key & 15) * 128 + (((ch & 7) ^ (key & 7)) << 4)), dst[j2]);
         }
       };
       load_k(0, kf[0]);
@@ -666,7 +666,7 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
         for (int dd = 0; dd < DG; ++dd) {
           const int key = j * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
           const int ch = (d0 + dd) * 2 + (lane >> 4);
-          ldmatrix_x4_trans(smem_u32(vt + (key >> 4) * 2 * PAGE_BYTES + (key & 15) * ROWB + ((ch ^ (key & 7)) << 4)), dst[dd]);
+          ldmatrix_x4_trans(smem_u32(vt + (key >> 4) * 2 * PAGE_BYTES + (ch >> 3) * 2048 + (key & 15) * 128 + (((ch & 7) ^ (key & 7)) << 4)), dst[dd]);
         }
       };
       load_v(0, vf[0]);
@@ -741,6 +741,369 @@ attention_rows(const AttnTcArgs a, unsigned long long* tr) {
 #pragma unroll
     for (int d = 0; d < HD / 8; ++d)
       *reinterpret_cast<uint32_t*>(po + d * 8 + (lane & 3) * 2) = pack_bf16(o[d][2 * r] * inv, o[d][2 * r + 1] * inv);
+  }
+}
+
+// ------------------------------------------------------------------ long contexts: shared K/V tiles, split keys
+// At thousands of cached positions the kernel above reads a head's K/V once per 16-row block (four
+// times at 64 tree rows) and keeps only six warps on an SM. Here a CTA owns up to 64 query rows of one
+// head (AS_RB blocks of 16) and one split of the keys, with AS_RB x AS_KP warps: warp (rb, kp) works on
+// rows [16 rb, +16) and on every AS_KP-th sub-tile of 32 keys of the split. The AS_RB warps of a key
+// phase share a ring of AS_NB sub-tile buffers (full / empty mbarriers per buffer, no CTA-wide barrier in
+// the loop): lane 0 of the phase's first warp refills a buffer once all of the phase's warps have
+// released it. K/V therefore reach the SM once per 64 rows, and twelve warps hide each other's MMA and
+// softmax latencies. The key phases are merged through shared memory, the splits by the CTA that arrives
+// last (as in attention_tc). Grid (heads, splits, sequences x row halves); the splits in use and their
+// sub-tiles follow from the sequence length on the device.
+constexpr int AS_RB = 4, AS_KP = 3, AS_NB = 4;
+constexpr int AS_SPLIT_SUB = 16;              // fewest sub-tiles worth a split of their own
+
+__host__ __device__ inline size_t attention_shared_smem(int head_dim) {
+  const size_t rowb = (size_t)head_dim * 2;
+  return AS_RB * 16 * rowb + (size_t)AS_KP * AS_NB * 2 * 32 * rowb + 8 * (size_t)(2 * AS_KP * AS_NB) + 4 * ATTN_PT_CACHE;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(AS_RB * AS_KP * 32, 1)
+attention_shared(const AttnTcArgs a, unsigned long long* tr) {
+  KTrace kt(tr);
+  constexpr int SK = 32;                      // keys per sub-tile
+  constexpr int ROWB = HD * 2;
+  constexpr int SUB_BYTES = SK * ROWB;        // one operand of a sub-tile
+  constexpr int PAGE_BYTES = 16 * ROWB;
+  constexpr int NTHR = AS_RB * AS_KP * 32;
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* qs = smem;                                                              // [AS_RB*16][HD]
+  uint8_t* kv = qs + AS_RB * 16 * ROWB;                                            // [AS_KP][AS_NB][page][K | V][16][HD]
+  uint64_t* full = reinterpret_cast<uint64_t*>(kv + AS_KP * AS_NB * 2 * SUB_BYTES);  // [AS_KP][AS_NB]
+  uint64_t* empty = full + AS_KP * AS_NB;                                          // [AS_KP][AS_NB]
+  int* pt_s = reinterpret_cast<int*>(empty + AS_KP * AS_NB);                       // [ATTN_PT_CACHE]
+
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rb = warp % AS_RB, kp = warp / AS_RB;
+  const int halves = gridDim.z / a.rows.B;
+  const int h = blockIdx.x, sp = blockIdx.y, b = blockIdx.z / halves, half = blockIdx.z % halves;
+  const int row0 = half * (AS_RB * 16);
+  const int H = a.H, kvh = h / (H / a.g.n_kv_heads);
+  const int* pt = a.page_table + b * a.g.pages_per_seq;
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  const int R = a.rows.R, cnt = a.rows.cnt[b], n = a.rows.n[b];
+  const int S = n + cnt, M = a.rows.B * R;
+  const int n_sub = (S + SK - 1) / SK;
+  const int nsplit = max(1, min(a.nsplit, (n_sub + AS_SPLIT_SUB - 1) / AS_SPLIT_SUB));
+  const int sps = (n_sub + nsplit - 1) / nsplit;
+  const int st0 = sp * sps, st1 = min(n_sub, st0 + sps);
+  if (row0 >= cnt || sp >= nsplit) return;                        // nothing in flight yet
+  const int nrb = min(AS_RB, (cnt - row0 + 15) >> 4);              // row blocks with a valid row
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < AS_KP * AS_NB; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], nrb); }
+    mbar_fence_init();
+  }
+  for (int e = threadIdx.x; e < ATTN_PT_CACHE; e += NTHR) {
+    const int idx = st0 * (SK / 16) + e;
+    pt_s[e] = idx < a.g.pages_per_seq ? pt[idx] : 0;
+  }
+  // Q tile of the CTA's rows (rows beyond cnt hold zeros)
+  const int i0 = row0 + rb * 16 + (lane >> 2), i1 = i0 + 8;    // this thread's two query rows
+  uint32_t anc0[4], anc1[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) { anc0[w] = i0 < cnt ? a.rows.anc[i0 * 4 + w] : 0u; anc1[w] = i1 < cnt ? a.rows.anc[i1 * 4 + w] : 0u; }
+  constexpr int QC = AS_RB * 16 * (HD / 8);
+  for (int c = threadIdx.x; c < QC; c += NTHR) {
+    const int r = c / (HD / 8), ch = c % (HD / 8);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (row0 + r < cnt) v = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + row0 + r) * H * HD + h * HD + ch * 8);
+    *reinterpret_cast<uint4*>(qs + r * ROWB + ((ch ^ (r & 7)) << 4)) = v;
+  }
+  __syncthreads();   // barriers initialised, page entries and Q staged
+
+  uint8_t* ring = kv + (size_t)kp * AS_NB * 2 * SUB_BYTES;
+  uint64_t* my_full = full + kp * AS_NB;
+  uint64_t* my_empty = empty + kp * AS_NB;
+  const int my_count = st0 + kp < st1 ? (st1 - st0 - kp + AS_KP - 1) / AS_KP : 0;    // sub-tiles of this key phase
+  auto issue = [&](int idx) {                                  // lane 0 of the phase's first warp
+    const int st = st0 + kp + idx * AS_KP, bf = idx % AS_NB;
+    mbar_expect_tx(&my_full[bf], 2 * SUB_BYTES);
+#pragma unroll
+    for (int pg = 0; pg < SK / 16; ++pg) {
+      const int e = (st - st0) * (SK / 16) + pg;
+      const int page = e < ATTN_PT_CACHE ? pt_s[e] : pt[st * (SK / 16) + pg];
+      bulk_load_1d(ring + bf * 2 * SUB_BYTES + pg * 2 * PAGE_BYTES, a.pool + a.g.block_offset(page, a.layer, 0, kvh), 2 * PAGE_BYTES, &my_full[bf]);
+    }
+  };
+  bool ok = true;
+  int issued = 0;
+  float o[HD / 8][4];
+#pragma unroll
+  for (int d = 0; d < HD / 8; ++d) o[d][0] = o[d][1] = o[d][2] = o[d][3] = 0.f;
+  float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
+  if (rb < nrb) {
+    uint32_t qf[HD / 16][4];
+    {
+      const int row = rb * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+      for (int kk = 0; kk < HD / 16; ++kk) {
+        const int ch = kk * 2 + (lane >> 4);
+        ldmatrix_x4(smem_u32(qs + row * ROWB + ((ch ^ (row & 7)) << 4)), qf[kk]);
+      }
+    }
+    for (int j = 0; j < my_count; ++j) {
+      const int bf = j % AS_NB;
+      if (rb == 0) {
+        // keep AS_NB sub-tiles of this phase in flight: a buffer is refilled once every warp of the phase released it
+        const int upto = min(j + AS_NB, my_count);
+        while (issued < upto && ok) {
+          if (issued >= AS_NB && !mbar_wait(&my_empty[issued % AS_NB], ((issued / AS_NB) - 1) & 1, a.status, 23)) { ok = false; break; }
+          if (lane == 0) issue(issued);
+          ++issued;
+        }
+        if (!ok) break;
+      }
+      if (!mbar_wait(&my_full[bf], (j / AS_NB) & 1, a.status, 20)) { ok = false; break; }
+      const int st = st0 + kp + j * AS_KP;
+      if (st == 0 && rb == 0 && lane == 0) trace_mark_max(tr, 3);
+      const uint8_t* ktile = ring + bf * 2 * SUB_BYTES;     // key `key` of the sub-tile: page key / 16, row key % 16
+      const uint8_t* vtile = ktile + PAGE_BYTES;
+      float s[SK / 8][4];
+#pragma unroll
+      for (int jj = 0; jj < SK / 8; ++jj) s[jj][0] = s[jj][1] = s[jj][2] = s[jj][3] = 0.f;
+      {
+        uint32_t kf[2][SK / 16][4];
+        auto load_k = [&](int kk, uint32_t (&dst)[SK / 16][4]) {
+#pragma unroll
+          for (int j2 = 0; j2 < SK / 16; ++j2) {
+            const int key = j2 * 16 + (lane & 7) + (lane >> 4) * 8;
+            const int ch = kk * 2 + ((lane >> 3) & 1);
+            ldmatrix_x4(smem_u32(ktile + (key >> 4) * 2 * PAGE_BYTES + (ch >> 3) * 2048 + (key & 15) * 128 + (((ch & 7) ^ (key & 7)) << 4)), dst[j2]);
+          }
+        };
+        load_k(0, kf[0]);
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          if (kk + 1 < HD / 16) load_k(kk + 1, kf[(kk + 1) & 1]);
+#pragma unroll
+          for (int j2 = 0; j2 < SK / 16; ++j2) {
+            mma_bf16_16816(s[2 * j2], qf[kk], kf[kk & 1][j2][0], kf[kk & 1][j2][1]);
+            mma_bf16_16816(s[2 * j2 + 1], qf[kk], kf[kk & 1][j2][2], kf[kk & 1][j2][3]);
+          }
+        }
+      }
+      const int k0 = st * SK;
+      float tmax[2] = {-INFINITY, -INFINITY};
+      if (k0 + SK > n) {
+        const uint32_t vis0 = (uint32_t)attn_vis64(anc0, k0, n), vis1 = (uint32_t)attn_vis64(anc1, k0, n);
+#pragma unroll
+        for (int jj = 0; jj < SK / 8; ++jj) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float v = s[jj][e] * a.scale_log2;
+            const int bi = jj * 8 + (lane & 3) * 2 + (e & 1);
+            if (!(((e < 2 ? vis0 : vis1) >> bi) & 1u)) v = -INFINITY;
+            s[jj][e] = v;
+            tmax[e >> 1] = fmaxf(tmax[e >> 1], v);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int jj = 0; jj < SK / 8; ++jj) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            s[jj][e] *= a.scale_log2;
+            tmax[e >> 1] = fmaxf(tmax[e >> 1], s[jj][e]);
+          }
+        }
+      }
+      float alpha[2], mnew[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 1));
+        tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 2));
+        mnew[r] = fmaxf(mrow[r], tmax[r]);
+        const float base = (mnew[r] == -INFINITY) ? 0.f : mnew[r];
+        alpha[r] = exp2f(mrow[r] - base);
+        mrow[r] = mnew[r];
+        mnew[r] = base;
+        lrow[r] *= alpha[r];
+      }
+#pragma unroll
+      for (int d = 0; d < HD / 8; ++d) { o[d][0] *= alpha[0]; o[d][1] *= alpha[0]; o[d][2] *= alpha[1]; o[d][3] *= alpha[1]; }
+      uint32_t pf[SK / 16][4];
+#pragma unroll
+      for (int jj = 0; jj < SK / 8; ++jj) {
+        const float p0 = exp2f(s[jj][0] - mnew[0]), p1 = exp2f(s[jj][1] - mnew[0]);
+        const float p2 = exp2f(s[jj][2] - mnew[1]), p3 = exp2f(s[jj][3] - mnew[1]);
+        lrow[0] += p0 + p1;
+        lrow[1] += p2 + p3;
+        pf[jj >> 1][(jj & 1) * 2 + 0] = pack_bf16(p0, p1);
+        pf[jj >> 1][(jj & 1) * 2 + 1] = pack_bf16(p2, p3);
+      }
+      {
+        constexpr int DG = 4, NG = (SK / 16) * (HD / 16) / DG;
+        uint32_t vf[2][DG][4];
+        auto load_v = [&](int g, uint32_t (&dst)[DG][4]) {
+          const int jv = g / (HD / 16 / DG), d0 = (g % (HD / 16 / DG)) * DG;
+#pragma unroll
+          for (int dd = 0; dd < DG; ++dd) {
+            const int key = jv * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            const int ch = (d0 + dd) * 2 + (lane >> 4);
+            ldmatrix_x4_trans(smem_u32(vtile + (key >> 4) * 2 * PAGE_BYTES + (ch >> 3) * 2048 + (key & 15) * 128 + (((ch & 7) ^ (key & 7)) << 4)), dst[dd]);
+          }
+        };
+        load_v(0, vf[0]);
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          if (g + 1 < NG) load_v(g + 1, vf[(g + 1) & 1]);
+          const int jv = g / (HD / 16 / DG), d0 = (g % (HD / 16 / DG)) * DG;
+#pragma unroll
+          for (int dd = 0; dd < DG; ++dd) {
+            mma_bf16_16816(o[2 * (d0 + dd)], pf[jv], vf[g & 1][dd][0], vf[g & 1][dd][1]);
+            mma_bf16_16816(o[2 * (d0 + dd) + 1], pf[jv], vf[g & 1][dd][2], vf[g & 1][dd][3]);
+          }
+        }
+      }
+      __syncwarp();                              // every lane has read the buffer
+      if (lane == 0) mbar_arrive(&my_empty[bf]);
+    }
+    if (!ok && rb == 0 && lane == 0) {
+      // a wait gave up: copies this phase may still have in flight get a bounded time to land
+      for (int i = issued > AS_NB ? issued - AS_NB : 0; i < issued; ++i) mbar_wait(&my_full[i % AS_NB], (i / AS_NB) & 1, a.status, 22);
+    }
+  }
+  ok = __syncthreads_and(ok);                    // all warps are done with the buffers
+  if (!ok) return;
+
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
+  }
+  // merge the key phases of a row block through the (now idle) K/V buffers: phases 1.. leave their state,
+  // phase 0 adds them in phase order
+  float* ex = reinterpret_cast<float*>(kv);
+  constexpr int SLOT = (HD / 2 + 4) * 32;       // floats per warp state
+  if (kp > 0 && rb < nrb) {
+    float* my = ex + (size_t)((kp - 1) * AS_RB + rb) * SLOT;
+#pragma unroll
+    for (int d = 0; d < HD / 8; ++d)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) my[(d * 4 + e) * 32 + lane] = o[d][e];
+    my[(HD / 2 + 0) * 32 + lane] = mrow[0]; my[(HD / 2 + 1) * 32 + lane] = mrow[1];
+    my[(HD / 2 + 2) * 32 + lane] = lrow[0]; my[(HD / 2 + 3) * 32 + lane] = lrow[1];
+  }
+  __syncthreads();
+  if (kp == 0 && rb < nrb) {
+#pragma unroll 1
+    for (int g2 = 1; g2 < AS_KP; ++g2) {
+      const float* th = ex + (size_t)((g2 - 1) * AS_RB + rb) * SLOT;
+      float w0[2], w1[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const float m1 = th[(HD / 2 + r) * 32 + lane], l1 = th[(HD / 2 + 2 + r) * 32 + lane];
+        const float mm = fmaxf(mrow[r], m1);
+        const float base = (mm == -INFINITY) ? 0.f : mm;
+        w0[r] = exp2f(mrow[r] - base);
+        w1[r] = exp2f(m1 - base);
+        mrow[r] = mm;
+        lrow[r] = lrow[r] * w0[r] + l1 * w1[r];
+      }
+#pragma unroll
+      for (int d = 0; d < HD / 8; ++d)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[d][e] = o[d][e] * w0[e >> 1] + th[(d * 4 + e) * 32 + lane] * w1[e >> 1];
+    }
+    if (nsplit == 1) {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int i = r ? i1 : i0;
+        if (i >= cnt) continue;
+        const float inv = 1.f / lrow[r];
+        bf16* po = a.out + ((size_t)b * R + i) * H * HD + h * HD;
+#pragma unroll
+        for (int d = 0; d < HD / 8; ++d)
+          *reinterpret_cast<uint32_t*>(po + d * 8 + (lane & 3) * 2) = pack_bf16(o[d][2 * r] * inv, o[d][2 * r + 1] * inv);
+      }
+    } else {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int i = r ? i1 : i0;
+        if (i >= cnt) continue;
+        const size_t m = (size_t)b * R + i;
+        float* po = a.part_o + ((size_t)sp * M + m) * H * HD + h * HD;
+#pragma unroll
+        for (int d = 0; d < HD / 8; ++d)
+          *reinterpret_cast<float2*>(po + d * 8 + (lane & 3) * 2) = make_float2(o[d][2 * r], o[d][2 * r + 1]);
+        if ((lane & 3) == 0) {
+          float* ml = a.part_ml + (((size_t)sp * M + m) * H + h) * 2;
+          ml[0] = mrow[r];
+          ml[1] = lrow[r];
+        }
+      }
+    }
+  }
+  if (nsplit == 1) return;
+  // the CTA of this (sequence, row half, head) that arrives last merges the splits
+  __shared__ int last_s;
+  __threadfence();
+  __syncthreads();
+  unsigned int* ctr = a.arrive + ((size_t)b * halves + half) * H + h;
+  if (threadIdx.x == 0) {
+    const unsigned int old = atomicAdd(ctr, 1u);
+    const int last = (old == (unsigned int)(nsplit - 1)) ? 1 : 0;
+    if (last) *ctr = 0u;
+    last_s = last;
+  }
+  __syncthreads();
+  if (!last_s) return;
+  __threadfence();
+  {
+    // two threads per query row, each merging half of the head dimension
+    const int il = threadIdx.x >> 1, d0 = (threadIdx.x & 1) * (HD / 2);
+    const int i = row0 + il;
+    if (il < AS_RB * 16 && i < cnt) {
+      const size_t m = (size_t)b * R + i;
+      float wgt[16];
+      float mx = -INFINITY, L = 0.f;
+#pragma unroll
+      for (int s2 = 0; s2 < 16; ++s2) {
+        wgt[s2] = -INFINITY;
+        if (s2 < nsplit) wgt[s2] = __ldcg(a.part_ml + (((size_t)s2 * M + m) * H + h) * 2);
+        mx = fmaxf(mx, wgt[s2]);
+      }
+#pragma unroll
+      for (int s2 = 0; s2 < 16; ++s2)
+        if (s2 < nsplit) {
+          const float l2 = __ldcg(a.part_ml + (((size_t)s2 * M + m) * H + h) * 2 + 1);
+          wgt[s2] = exp2f(wgt[s2] - mx);
+          L += wgt[s2] * l2;
+        }
+      float acc[HD / 2];
+#pragma unroll
+      for (int e = 0; e < HD / 2; ++e) acc[e] = 0.f;
+#pragma unroll
+      for (int s2 = 0; s2 < 16; ++s2) {
+        if (s2 >= nsplit) break;
+        const float w = wgt[s2];
+        const float* src = a.part_o + ((size_t)s2 * M + m) * H * HD + h * HD + d0;
+        float4 v[HD / 8];
+#pragma unroll
+        for (int e = 0; e < HD / 8; ++e) v[e] = __ldcg(reinterpret_cast<const float4*>(src + e * 4));
+#pragma unroll
+        for (int e = 0; e < HD / 8; ++e) {
+          acc[4 * e] += w * v[e].x; acc[4 * e + 1] += w * v[e].y; acc[4 * e + 2] += w * v[e].z; acc[4 * e + 3] += w * v[e].w;
+        }
+      }
+      const float inv = 1.f / L;
+      bf16* dst = a.out + m * H * HD + h * HD + d0;
+#pragma unroll
+      for (int e = 0; e < HD / 8; ++e) {
+        uint2 pk;
+        pk.x = pack_bf16(acc[4 * e] * inv, acc[4 * e + 1] * inv);
+        pk.y = pack_bf16(acc[4 * e + 2] * inv, acc[4 * e + 3] * inv);
+        *reinterpret_cast<uint2*>(dst + e * 4) = pk;
+      }
+    }
   }
 }
 

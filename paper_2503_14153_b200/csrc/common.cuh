@@ -54,15 +54,19 @@ __device__ __forceinline__ void warp_argmax(float& v, int& i) {
 }
 
 // ------------------------------------------------------------------ KV page layout
-// Pool layout: [page][layer][kv_head][K|V][page_size rows][head_dim]: the K block and the V
-// block of a (page, layer, head) are adjacent, so one bulk copy brings both (a bulk copy costs
-// about the same whether it moves 4 KB or 8 KB). Within a block a row holds head_dim elements; 16-byte chunks of a row are
-// XOR-swizzled with the row index (low 3 bits) when a row is 256 bytes of bf16, so that a
-// plain bulk copy of the block lands in shared memory in a bank-conflict-free layout for
-// ldmatrix. float32 caches are stored unswizzled.
-template <typename T> __device__ __host__ __forceinline__ int kv_elem(int row, int d) { return d; }
-template <> __device__ __host__ __forceinline__ int kv_elem<bf16>(int row, int d) {
-  return ((((d >> 3) ^ (row & 7)) << 3) | (d & 7));
+// Pool layout: [page][layer][kv_head][K|V][block]: the K block and the V block of a (page, layer, head) are
+// adjacent, so one bulk copy brings both (a bulk copy costs about the same whether it moves 4 KB or 8 KB).
+// A float32 block is page_size rows of head_dim values. A bf16 block (head_dim % 64 == 0) holds head_dim / 64
+// slabs; slab h = dims [64 h, 64 h + 64) of all page_size rows, a row of a slab being 128 bytes whose eight
+// 16-byte chunks are XOR-swizzled with the row index (low 3 bits). That is the tensor cores' canonical K-major
+// tile with the 128-byte swizzle: slabs of consecutive pages appended in shared memory are a valid tcgen05.mma
+// operand as they are (K as the K-major B operand of Q K^T, V as the MN-major B operand of P V), and the rows are
+// conflict-free for ldmatrix. kv_elem returns the element offset of (row, d) relative to the row's nominal
+// base `block + row * head_dim` (it may be negative).
+template <typename T> __device__ __host__ __forceinline__ int kv_elem(int row, int d, int D, int ps) { return d; }
+template <> __device__ __host__ __forceinline__ int kv_elem<bf16>(int row, int d, int D, int ps) {
+  const int h = d >> 6, dd = d & 63;
+  return h * ps * 64 + row * 64 + ((((dd >> 3) ^ (row & 7)) << 3) | (dd & 7)) - row * D;
 }
 
 struct KVGeom {

@@ -200,8 +200,8 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
             const int slot = p.rows.slot[m];
             const int page = p.page_table[b * p.g.pages_per_seq + slot / p.g.page_size], prow = slot % p.g.page_size;
             // (a group of four lies inside one 16-byte chunk of the row: the chunk swizzle keeps it contiguous)
-            dst[k] = p.pool + p.g.block_offset(page, p.layer, rope_mat - 1, head) + (size_t)prow * D + kv_elem<bf16>(prow, i);
-            lo_c[k] |= (kv_elem<bf16>(prow, i + half) - kv_elem<bf16>(prow, i)) << 16;   // distance to the upper half's group
+            dst[k] = p.pool + p.g.block_offset(page, p.layer, rope_mat - 1, head) + (size_t)prow * D + kv_elem<bf16>(prow, i, D, p.g.page_size);
+            lo_c[k] |= (kv_elem<bf16>(prow, i + half, D, p.g.page_size) - kv_elem<bf16>(prow, i, D, p.g.page_size)) << 16;   // distance to the upper half's group
           }
         }
       }

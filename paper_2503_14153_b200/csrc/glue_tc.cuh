@@ -182,8 +182,8 @@ rope_store_tc(const PartView pv, int qp0, int kp0, int vp0, Rows rows, const flo
       } else {
         const int page = page_table[b * g.pages_per_seq + slot / g.page_size], prow = slot % g.page_size;
         bf16* dst = pool + g.block_offset(page, layer, 0, head - H) + (size_t)prow * D;
-        *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e)) = lo;
-        *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e + half)) = hi;
+        *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e, D, g.page_size)) = lo;
+        *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e + half, D, g.page_size)) = hi;
       }
     } else {
       const int iv = it - n_rot;
@@ -192,7 +192,7 @@ rope_store_tc(const PartView pv, int qp0, int kp0, int vp0, Rows rows, const flo
       if (i >= cnt) continue;
       const int page = page_table[b * g.pages_per_seq + slot / g.page_size], prow = slot % g.page_size;
       bf16* dst = pool + g.block_offset(page, layer, 1, kh) + (size_t)prow * D;
-      *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e)) = pack4_bf16(a.x, a.y, a.z, a.w);
+      *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e, D, g.page_size)) = pack4_bf16(a.x, a.y, a.z, a.w);
     }
   }
 }

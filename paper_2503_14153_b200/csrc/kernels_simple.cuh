@@ -230,8 +230,8 @@ __global__ void rope_store(const float* __restrict__ qkv, int nsplit, size_t spl
     } else {
       int kh = head - H;
       T* dst = pool + g.block_offset(page, layer, 0, kh) + (size_t)prow * D;
-      dst[kv_elem<T>(prow, e)] = from_f<T>(r0);
-      dst[kv_elem<T>(prow, e + half)] = from_f<T>(r1);
+      dst[kv_elem<T>(prow, e, D, g.page_size)] = from_f<T>(r0);
+      dst[kv_elem<T>(prow, e + half, D, g.page_size)] = from_f<T>(r1);
     }
   }
   for (int p = threadIdx.x; p < nk; p += blockDim.x) {
@@ -239,7 +239,7 @@ __global__ void rope_store(const float* __restrict__ qkv, int nsplit, size_t spl
     float a = 0.f;
     for (int s = 0; s < max(nsplit, 1); ++s) a += src[s * split_stride + nq + nk + p];
     T* dst = pool + g.block_offset(page, layer, 1, kh) + (size_t)prow * D;
-    dst[kv_elem<T>(prow, e)] = from_f<T>(a);
+    dst[kv_elem<T>(prow, e, D, g.page_size)] = from_f<T>(a);
   }
 }
 
@@ -270,7 +270,7 @@ __global__ void attention_simple(const T* __restrict__ q, T* __restrict__ out, c
     int prow = j % g.page_size;
     const T* kr = pool + g.block_offset(pt[j / g.page_size], layer, 0, kvh) + (size_t)prow * D;
     float s = 0.f;
-    for (int e = 0; e < EPL; ++e) s = fmaf(qv[e], to_f<T>(kr[kv_elem<T>(prow, lane * EPL + e)]), s);
+    for (int e = 0; e < EPL; ++e) s = fmaf(qv[e], to_f<T>(kr[kv_elem<T>(prow, lane * EPL + e, D, g.page_size)]), s);
     s = warp_sum(s) * scale;
     mx = fmaxf(mx, s);
   }
@@ -283,12 +283,12 @@ __global__ void attention_simple(const T* __restrict__ q, T* __restrict__ out, c
     const T* kr = pool + g.block_offset(page, layer, 0, kvh) + (size_t)prow * D;
     const T* vr = pool + g.block_offset(page, layer, 1, kvh) + (size_t)prow * D;
     float s = 0.f;
-    for (int e = 0; e < EPL; ++e) s = fmaf(qv[e], to_f<T>(kr[kv_elem<T>(prow, lane * EPL + e)]), s);
+    for (int e = 0; e < EPL; ++e) s = fmaf(qv[e], to_f<T>(kr[kv_elem<T>(prow, lane * EPL + e, D, g.page_size)]), s);
     s = warp_sum(s) * scale;
     float p = expf(s - mx);
     l += p;
     float pq = quant<T>(p);
-    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pq, to_f<T>(vr[kv_elem<T>(prow, lane * EPL + e)]), acc[e]);
+    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pq, to_f<T>(vr[kv_elem<T>(prow, lane * EPL + e, D, g.page_size)]), acc[e]);
   }
   float inv = 1.f / l;
   for (int e = 0; e < EPL; ++e) out[(size_t)m * H * D + h * D + lane * EPL + e] = from_f<T>(acc[e] * inv);
@@ -640,7 +640,7 @@ __global__ void compact_kv(T* __restrict__ pool, KVGeom g, const int* __restrict
     int sr = src % g.page_size, dr = dst % g.page_size;
     const T* s = pool + g.block_offset(pt[src / g.page_size], lk >> 1, lk & 1, head) + (size_t)sr * D;
     T* t = pool + g.block_offset(pt[dst / g.page_size], lk >> 1, lk & 1, head) + (size_t)dr * D;
-    for (int e = threadIdx.x; e < D; e += blockDim.x) t[kv_elem<T>(dr, e)] = s[kv_elem<T>(sr, e)];
+    for (int e = threadIdx.x; e < D; e += blockDim.x) t[kv_elem<T>(dr, e, D, g.page_size)] = s[kv_elem<T>(sr, e, D, g.page_size)];
   }
 }
 

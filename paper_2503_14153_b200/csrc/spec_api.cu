@@ -18,6 +18,7 @@
 #include <vector>
 
 #include "attention_tc.cuh"
+#include "attention_umma.cuh"
 #include "common.cuh"
 #include "gemm_cluster.cuh"
 #include "gemm_stream.cuh"
@@ -40,6 +41,7 @@ constexpr int MAX_STEPS_AHEAD = 8;      // enqueue-only steps the host may run a
 constexpr int ATTN_ROWS_WARPS = 6;      // warps of the CTA-per-16-rows attention kernel
 constexpr int ATTN_SPLIT_TILES = 8;       // fewest KV tiles a split of attention_tc gets (2..8 measured alike)
 constexpr int ATTN_SINGLE_TILES = 12;   // contexts of at most this many 64-key tiles use one KV split
+constexpr int ATTN_LONG_KEYS = 2048;    // default context length from which passes of more than 32 rows use the shared-K/V kernel
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -200,6 +202,10 @@ struct spec_ctx {
   int gemm_ctas = 288;                 // persistent CTAs of the weight-streaming GEMM (measured best; at most SM_SLOTS)
   int l2_prefetch = 0;
   bool gc_attr_set[12] = {};            // per context (and so per device): shared-memory attribute of each gemm_cluster instance set
+  int long_attn_keys = ATTN_LONG_KEYS; // SPEC_OPT_LONG_ATTN_KEYS (0 = never)
+  bool attn_umma = true;               // SPEC_OPT_ATTN_UMMA: the long-context kernel is the tcgen05 one (head_dim 128)
+  CUtensorMap tm_kv;                   // 5-D view of the page pool for its TMA loads
+  bool tm_kv_ok = false;
   bool wide_gemm = true;               // SPEC_OPT_WIDE_GEMM: passes of more than 128 rows use the 128 x 256-tile kernel
   int cluster_epilogue = 2;            // SPEC_OPT_CLUSTER_EPILOGUE: which projections finish their split-K sums inside a cluster
                                        // (bits: 1 output/down, 2 gate+up, 4 q/k/v; measured on the 7B shape: only gate+up pays)
@@ -347,7 +353,7 @@ size_t carve(spec_ctx* c, void* base) {
 
   c->d_status = b.take<int>(4);
   c->d_trace = b.take<unsigned long long>((size_t)TRACE_CAP * 4);
-  c->d_attn_arrive = b.take<unsigned int>((size_t)B * f.n_heads);
+  c->d_attn_arrive = b.take<unsigned int>((size_t)B * f.n_heads * 2);
   c->d_pval2 = b.take<float>(c->Mcap); c->d_pidx2 = b.take<int>(c->Mcap);
   c->d_draws = b.take<int>(B);
   c->d_n = b.take<int>(B); c->d_cnt = b.take<int>(B); c->d_n_old = b.take<int>(B); c->d_root = b.take<int>(B);
@@ -664,6 +670,12 @@ bool attn_rows_mode(const spec_ctx* c, int R) {
   return nw > 1 && c->cfg.n_heads * c->B * nw <= SM_SLOTS / 2;
 }
 
+// Passes of more than 32 rows over a context that may reach long_attn_keys positions.
+bool attn_long_mode(const spec_ctx* c, int R, int keys_hi) {
+  const bool umma = c->attn_umma && c->tm_kv_ok && c->cfg.head_dim == 128;
+  return c->long_attn_keys > 0 && (R > 32 || umma) && keys_hi > c->long_attn_keys;
+}
+
 // n_hi_pass / n_lo_pass: host bounds of the cached length the pass's rows sit on, per sequence
 // (n_lo_pass may be null: nothing is fetched before the dependency wait).
 int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* n_hi_pass, const int* n_lo_pass) {
@@ -681,6 +693,38 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
     if (b < ATTN_MAX_SEQS) a.n_lo[b] = n_lo_pass ? n_lo_pass[b] : 0;
   }
   const int nw = (R + 15) / 16;
+  if (attn_long_mode(c, R, tiles_hi * 64) && c->attn_umma && c->tm_kv_ok && D == 128) {
+    // long contexts: scores and P V on tcgen05, a CTA per (head, 64 rows, key split)
+    const int halves = (R + AU_ROWS - 1) / AU_ROWS;
+    a.nsplit = std::max(1, std::min(c->nsplit_attn, (SM_SLOTS / 2) / (H * c->B * halves)));
+    dim3 grid(H, a.nsplit, c->B * halves);
+    ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
+    static bool set_dev[kAttrDevices] = {};
+    bool& set_ = *attr_flag(set_dev);
+    if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_umma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_umma_smem())); set_ = true; }
+    cudaError_t e_ = launch_k(c->pdl, attention_umma<128>, grid, dim3(AU_THREADS), attention_umma_smem(), c->stream, c->tm_kv, a, c->next_trace("attention_tc"));
+    c->launches++;
+    if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("attention_umma: ") + cudaGetErrorString(e_));
+    return SPEC_OK;
+  }
+  if (attn_long_mode(c, R, tiles_hi * 64) && R > 32) {
+    // long contexts, more than 32 rows: K/V tiles shared by the row blocks of a CTA, keys split across CTAs
+    const int halves = (R + AS_RB * 16 - 1) / (AS_RB * 16);
+    a.nsplit = std::max(1, std::min(c->nsplit_attn, (SM_SLOTS / 2) / (H * c->B * halves)));
+    a.stages = AS_NB; a.split_tiles = AS_SPLIT_SUB;
+    dim3 grid(H, a.nsplit, c->B * halves);
+    ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
+    static bool set_dev[2][kAttrDevices] = {};
+    bool& set_ = *attr_flag(set_dev[D == 128 ? 0 : 1]);
+    if (D == 128) {
+      if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_shared<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_shared_smem(128))); set_ = true; }
+      KLAUNCH("attention_tc", (attention_shared<128>), grid, dim3(AS_RB * AS_KP * 32), attention_shared_smem(128), a);
+    } else {
+      if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_shared<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_shared_smem(64))); set_ = true; }
+      KLAUNCH("attention_tc", (attention_shared<64>), grid, dim3(AS_RB * AS_KP * 32), attention_shared_smem(64), a);
+    }
+    return SPEC_OK;
+  }
   if (attn_rows_mode(c, R)) {
     // few sequences: a CTA per (head, 16 query rows) walks the whole context, whatever its length
     a.nsplit = 1; a.stages = 2; a.split_tiles = 1;
@@ -1077,8 +1121,15 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
   // length bounds and a recorded step serves every length below its bound
   std::vector<int> n_hi_plan(B), n_lo_plan(B);
   for (int b = 0; b < B; ++b) {
-    const bool any_len = attn_rows_mode(c, T_) || c->n_hi[b] + T_ > ATTN_SINGLE_TILES * 64;
-    n_hi_plan[b] = (any_len ? c->cap : std::min(ATTN_SINGLE_TILES * 64, c->cap)) - T_;
+    // three launch shapes: contexts that may reach the long-context kernel's threshold are planned for any length;
+    // below it the CTA-per-16-rows kernel serves every length up to the threshold, and the split kernel is planned
+    // for at most ATTN_SINGLE_TILES tiles or for any length
+    int bound;
+    if (attn_long_mode(c, T_, c->n_hi[b] + T_)) bound = c->cap;
+    else if (attn_rows_mode(c, T_)) bound = attn_long_mode(c, T_, 1 << 30) ? std::min(c->long_attn_keys / 64 * 64, c->cap) : c->cap;
+    else if (c->n_hi[b] + T_ > ATTN_SINGLE_TILES * 64) bound = attn_long_mode(c, T_, 1 << 30) ? std::min(std::max(c->long_attn_keys / 64 * 64, ATTN_SINGLE_TILES * 64), c->cap) : c->cap;
+    else bound = std::min(ATTN_SINGLE_TILES * 64, c->cap);
+    n_hi_plan[b] = bound - T_;
     n_lo_plan[b] = c->n_lo[b];
   }
   const bool use_graph = c->graph_on && !c->trace_on && c->profile_kind == 0;
@@ -1255,13 +1306,26 @@ int spec_create(const spec_config* cfg, const spec_weights* w, const spec_tree* 
   up(c->d_mw, c->mw.data(), c->mw.size() * sizeof(void*));
   up(c->d_mb, c->mb.data(), c->mb.size() * sizeof(void*));
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 4 * sizeof(int), c->stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_attn_arrive, 0, (size_t)cfg->max_batch * cfg->n_heads * sizeof(unsigned int), c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_attn_arrive, 0, (size_t)cfg->max_batch * cfg->n_heads * 2 * sizeof(unsigned int), c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_cand, 0, (size_t)cfg->max_batch * (c->K + 1) * c->kmax * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) { g_create_error = std::string("set-up copies: ") + cudaGetErrorString(e); delete c; return SPEC_E_CUDA; }
   if (cudaHostAlloc(reinterpret_cast<void**>(&c->h_n_pinned), (size_t)cfg->max_batch * sizeof(int), cudaHostAllocDefault) != cudaSuccess) c->h_n_pinned = nullptr;
   if (cudaEventCreateWithFlags(&c->n_ev, cudaEventDisableTiming) != cudaSuccess) c->n_ev = nullptr;
   cudaGetLastError();
+  if (c->tc && cfg->head_dim == 128 && cfg->page_size == 16) {
+    // 5-D view of the page pool for the tcgen05 attention: (64 dims of a slab row, 16 rows, slab index =
+    // ((layer * kv_heads + head) * 2 + K|V) * 2 + dims half, sequence, page); page p of sequence b is pool
+    // page p * max_batch + b (the table written above), so both are strided dimensions
+    EncodeTiledFn fn = get_encode_fn();
+    const cuuint64_t page_bytes = (cuuint64_t)c->geom.page_elems() * 2;
+    cuuint64_t dims[5] = {64, 16, (cuuint64_t)cfg->n_layers * cfg->n_kv_heads * 4, (cuuint64_t)cfg->max_batch, (cuuint64_t)c->pages_per_seq};
+    cuuint64_t strides[4] = {128, 2048, page_bytes, page_bytes * (cuuint64_t)cfg->max_batch};
+    cuuint32_t box[5] = {64, 16, 1, 1, AU_KT / 16};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    c->tm_kv_ok = fn && fn(&c->tm_kv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, c->d_pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  }
   *out = c;
   return SPEC_OK;
 }
@@ -1327,6 +1391,7 @@ int64_t spec_query(const spec_ctx* c, int32_t what) {
     case SPEC_Q_N_NODES: return c->T;
     case SPEC_Q_BATCH: return c->B;
     case SPEC_Q_GRAPH_CAPTURES: return c->graph_captures;
+    case SPEC_Q_WIDE_GEMM: return c->tc && c->wide_gemm ? 1 : 0;
     case SPEC_Q_CLUSTER_GATE_UP: return c->tc && cluster_gemm_ok(c, GC_SWIGLU, c->B * c->T, f.d_model) ? 1 : 0;
     case SPEC_Q_ALGO_BYTES_PER_STEP: {
       double d = f.d_model, F = f.d_ffn, V = f.vocab, HD = (double)f.n_heads * f.head_dim, KD = (double)f.n_kv_heads * f.head_dim;
@@ -1347,7 +1412,10 @@ int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
     case SPEC_OPT_L2_PREFETCH:
       if (value < 0 || value > 64) return c->fail(SPEC_E_BADARG, "L2 prefetch depth out of range");
       break;
-    case SPEC_OPT_GRAPH: case SPEC_OPT_PHASE_TIMING: case SPEC_OPT_PDL: case SPEC_OPT_TRACE: case SPEC_OPT_CLUSTER_EPILOGUE: case SPEC_OPT_WIDE_GEMM: break;
+    case SPEC_OPT_GRAPH: case SPEC_OPT_PHASE_TIMING: case SPEC_OPT_PDL: case SPEC_OPT_TRACE: case SPEC_OPT_CLUSTER_EPILOGUE: case SPEC_OPT_WIDE_GEMM: case SPEC_OPT_ATTN_UMMA: break;
+    case SPEC_OPT_LONG_ATTN_KEYS:
+      if (value < 0) return c->fail(SPEC_E_BADARG, "context threshold must not be negative");
+      break;
     default: return c->fail(SPEC_E_BADARG, "unknown option");
   }
   c->graph_epoch++;   // the option is valid: a recorded step no longer matches the options
@@ -1368,6 +1436,8 @@ int spec_set_option(spec_ctx* c, int32_t what, int32_t value) {
       c->small_gemm_ctas = value; return SPEC_OK;
     case SPEC_OPT_CLUSTER_EPILOGUE: c->cluster_epilogue = value & 7; return SPEC_OK;
     case SPEC_OPT_WIDE_GEMM: c->wide_gemm = value != 0; return SPEC_OK;
+    case SPEC_OPT_LONG_ATTN_KEYS: c->long_attn_keys = value; return SPEC_OK;
+    case SPEC_OPT_ATTN_UMMA: c->attn_umma = value != 0; return SPEC_OK;
     case SPEC_OPT_TRACE:
       c->trace_on = value != 0;
       if (c->trace_on && c->trace_init.empty()) {
@@ -1481,7 +1551,7 @@ int spec_debug_read_kv(spec_ctx* c, int32_t seq, int32_t layer, int32_t slot0, i
         for (int e = 0; e < D; ++e) {
           float v;
           if (c->esz == 2) {
-            uint16_t raw = reinterpret_cast<uint16_t*>(blk.data())[(size_t)row * D + kv_elem<bf16>(row, e)];
+            uint16_t raw = reinterpret_cast<uint16_t*>(blk.data())[(size_t)row * D + kv_elem<bf16>(row, e, D, ps)];
             uint32_t u32 = (uint32_t)raw << 16;
             memcpy(&v, &u32, 4);
           } else {

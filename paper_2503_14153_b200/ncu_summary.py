@@ -5,6 +5,10 @@
         [--traffic-kernel 'gemm_cluster<64,swiglu>' --match gemm_cluster --launch 1 --shape 4096 11008 64 \
          --sources paper_2503_14153_b200/csrc/gemm_cluster.cuh]
 
+    ncu --metrics gpu__time_duration.sum ... --csv --log-file launches.csv <cmd>
+    python -m paper_2503_14153_b200.ncu_summary launches.csv --launch-list --last-step-from medusa_act_tc \
+        --out profiles/NAME --command "..."
+
 Writes NAME.md (one row per captured launch: duration, DRAM bytes, DRAM and tensor-pipe utilisation,
 occupancy, registers) and, with --traffic-kernel, NAME.json holding the DRAM read + write bytes of
 one launch together with a hash of the kernel's source files: the benchmark reports that figure as
@@ -51,8 +55,32 @@ def parse(path):
     return out
 
 
+def launch_list(path, last_step_from):
+    """Per-kernel launches, total time and share of the launch list's last decode step (from the launch before
+    the last `last_step_from` kernel on) out of a `--metrics gpu__time_duration.sum --csv` log."""
+    lines = [l for l in open(path) if not l.startswith("==")]
+    seq = []
+    for row in csv.DictReader(lines):
+        if row.get("Metric Name") != "gpu__time_duration.sum":
+            continue
+        name = re.sub(r"^void\s+", "", re.sub(r"\(.*", "", row["Kernel Name"])).replace("spec::", "")
+        seq.append((name, to_number(row["Metric Value"], row["Metric Unit"]), row["Grid Size"]))
+    if last_step_from:
+        idx = [i for i, s in enumerate(seq) if last_step_from in s[0]]
+        if idx:
+            seq = seq[max(idx[-1] - 1, 0):]
+    agg = {}
+    for n, v, g in seq:
+        a = agg.setdefault(f"{n} {g}", [0, 0.0])
+        a[0] += 1
+        a[1] += v
+    return seq, agg
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--launch-list", action="store_true", help="the input is a gpu__time_duration launch list")
+    ap.add_argument("--last-step-from", default=None, help="keep the launches from the one before the last kernel of this name")
     ap.add_argument("raw_csv")
     ap.add_argument("--out", required=True, help="path prefix of the .md (and .json) to write")
     ap.add_argument("--command", required=True, help="the full command that made the capture")
@@ -63,6 +91,17 @@ def main():
     ap.add_argument("--shape", type=int, nargs="+", default=None)
     ap.add_argument("--sources", nargs="+", default=[])
     args = ap.parse_args()
+    if args.launch_list:
+        seq, agg = launch_list(args.raw_csv, args.last_step_from)
+        tot = sum(v for _, v, _ in seq)
+        with open(args.out + ".md", "w") as f:
+            f.write(f"# {args.title or os.path.basename(args.out)}\n\nCommand (B200, one GPU; the plain run exited 0 first):\n\n    {args.command}\n\n"
+                    f"Launches of the last captured decode step ({len(seq)} launches, {tot:.1f} us in all; times under the profiler are "
+                    "cold-cache and serialised: compare shares, not absolutes).\n\n")
+            f.write("| kernel grid | launches | total us | share | avg us |\n|---|---|---|---|---|\n")
+            for k, (c, t) in sorted(agg.items(), key=lambda x: -x[1][1]):
+                f.write(f"| {k} | {c} | {t:.1f} | {t / tot * 100:.1f}% | {t / c:.2f} |\n")
+        return
     launches = parse(args.raw_csv)
     with open(args.out + ".md", "w") as f:
         f.write(f"# {args.title or os.path.basename(args.out)}\n\nCommand (B200, one GPU; the plain run exited 0 first):\n\n    {args.command}\n\n")

@@ -108,6 +108,27 @@ def test_small_bf16_d512_cluster_epilogues(torch):
         assert r2.steps > 0
 
 
+@pytest.mark.parametrize("T,prompt_len,umma", [(64, 70, 1), (64, 700, 1), (128, 300, 1), (16, 150, 1), (32, 1100, 1),
+                                                (64, 700, 0), (128, 300, 0)])
+def test_long_context_attention_kernels_on_small_shapes(torch, T, prompt_len, umma):
+    """The long-context attention kernels (tcgen05 scores and P V with umma = 1, the shared-K/V mma.sync kernel with
+    umma = 0) forced onto short contexts by lowering their threshold to one position: one and several 128-key
+    tiles, key splits merged by the last CTA, two row halves at T = 128, trees of 16 and 32 rows, and prompt
+    processing in 128-row passes, all against the oracle."""
+    from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights
+    from paper_2503_14153_b200 import binding as B
+    from tests_lockstep import run_lockstep
+    cfg = SMALL_BF16_D128.with_(tree_nodes=T, seed=25)
+    w, prompt = draw_weights(cfg), draw_prompt(cfg, prompt_len)
+    tree = build_tree(cfg.topk, T)
+    gpu = SpecDecoder(cfg, upload_weights(cfg, w), tree, prompt_len + 40, flags=B.FLAG_KEEP_LOGITS)
+    gpu.set_option(B.OPT_ATTN_UMMA, umma)
+    gpu.set_option(B.OPT_LONG_ATTN_KEYS, 1)
+    rep = run_lockstep(cfg, w, tree, prompt, 12, TOL_BF16, TIE_GAP, gpu=gpu, check_kv_every=4)
+    gpu.close()
+    assert rep.steps > 0
+
+
 def test_ten_heads_deep_tree(torch):
     """The paper's head count (K = 10): ten stacked head matrices (three GEMM launches), a tree ten levels deep."""
     cfg = SMALL_BF16.with_(name="small_bf16_k10", n_medusa=10, topk=(4, 3, 2, 2, 2, 1, 1, 1, 1, 1), tree_nodes=48, seed=23)
