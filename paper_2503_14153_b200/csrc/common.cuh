@@ -54,8 +54,11 @@ __device__ __forceinline__ void warp_argmax(float& v, int& i) {
 }
 
 // ------------------------------------------------------------------ KV page layout
-// Pool layout: [page][layer][kv_head][K|V][block]: the K block and the V block of a (page, layer, head) are
-// adjacent, so one bulk copy brings both (a bulk copy costs about the same whether it moves 4 KB or 8 KB).
+// Pool layout: [layer][kv_head][page][K|V][block]. The K block and the V block of a (page, layer, head) are
+// adjacent, so one bulk copy brings both (a bulk copy costs about the same whether it moves 4 KB or 8 KB), and
+// the pages of one (layer, head) -- what an attention CTA streams -- lie side by side: with one sequence its
+// keys are one contiguous run of HBM, with several the runs interleave page by page (page p of sequence b is
+// pool page p * max_batch + b).
 // A float32 block is page_size rows of head_dim values. A bf16 block (head_dim % 64 == 0) holds head_dim / 64
 // slabs; slab h = dims [64 h, 64 h + 64) of all page_size rows, a row of a slab being 128 bytes whose eight
 // 16-byte chunks are XOR-swizzled with the row index (low 3 bits). That is the tensor cores' canonical K-major
@@ -76,8 +79,9 @@ struct KVGeom {
   __device__ __host__ __forceinline__ size_t page_elems() const {
     return (size_t)n_layers * 2 * n_kv_heads * block_elems();
   }
+  __device__ __host__ __forceinline__ size_t pool_pages() const { return (size_t)pages_per_seq * max_batch; }
   __device__ __host__ __forceinline__ size_t block_offset(int page, int layer, int kv, int head) const {
-    return (size_t)page * page_elems() + (((size_t)layer * n_kv_heads + head) * 2 + kv) * block_elems();
+    return ((((size_t)layer * n_kv_heads + head) * pool_pages() + page) * 2 + kv) * block_elems();
   }
 };
 

@@ -696,13 +696,29 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
   if (attn_long_mode(c, R, tiles_hi * 64) && c->attn_umma && c->tm_kv_ok && D == 128) {
     // long contexts: scores and P V on tcgen05, a CTA per (head, 64 rows, key split)
     const int halves = (R + AU_ROWS - 1) / AU_ROWS;
-    a.nsplit = std::max(1, std::min(c->nsplit_attn, (SM_SLOTS / 2) / (H * c->B * halves)));
+    // the key splits of a (sequence, row half, head) are one cluster: one CTA per SM, at most a wave of them
+    a.nsplit = std::max(1, std::min(std::min(c->nsplit_attn, AU_MAX_CLUSTER), (SM_SLOTS / 2) / (H * c->B * halves)));
     dim3 grid(H, a.nsplit, c->B * halves);
     ProfScope ps_attn(c, SPEC_PROFILE_ATTENTION);
     static bool set_dev[kAttrDevices] = {};
     bool& set_ = *attr_flag(set_dev);
     if (!set_) { CUDA_OK(cudaFuncSetAttribute(attention_umma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attention_umma_smem())); set_ = true; }
-    cudaError_t e_ = launch_k(c->pdl, attention_umma<128>, grid, dim3(AU_THREADS), attention_umma_smem(), c->stream, c->tm_kv, a, c->next_trace("attention_tc"));
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = dim3(AU_THREADS); cfg.dynamicSmemBytes = attention_umma_smem(); cfg.stream = c->stream;
+    cudaLaunchAttribute at[2];
+    int n_at = 0;
+    if (a.nsplit > 1) {
+      at[n_at].id = cudaLaunchAttributeClusterDimension;
+      at[n_at].val.clusterDim.x = 1; at[n_at].val.clusterDim.y = (unsigned)a.nsplit; at[n_at].val.clusterDim.z = 1;
+      ++n_at;
+    }
+    if (c->pdl) {
+      at[n_at].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      at[n_at].val.programmaticStreamSerializationAllowed = 1;
+      ++n_at;
+    }
+    cfg.attrs = at; cfg.numAttrs = (unsigned)n_at;
+    cudaError_t e_ = cudaLaunchKernelEx(&cfg, attention_umma<128>, c->tm_kv, a, c->next_trace("attention_tc"));
     c->launches++;
     if (e_ != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("attention_umma: ") + cudaGetErrorString(e_));
     return SPEC_OK;
@@ -1314,14 +1330,14 @@ int spec_create(const spec_config* cfg, const spec_weights* w, const spec_tree* 
   if (cudaEventCreateWithFlags(&c->n_ev, cudaEventDisableTiming) != cudaSuccess) c->n_ev = nullptr;
   cudaGetLastError();
   if (c->tc && cfg->head_dim == 128 && cfg->page_size == 16) {
-    // 5-D view of the page pool for the tcgen05 attention: (64 dims of a slab row, 16 rows, slab index =
-    // ((layer * kv_heads + head) * 2 + K|V) * 2 + dims half, sequence, page); page p of sequence b is pool
+    // 5-D view of the page pool for the tcgen05 attention: (64 dims of a slab row, the 64 slab rows of a page's
+    // K|V pair = 4 slabs x 16 rows, sequence, page, layer * kv_heads + head); page p of sequence b is pool
     // page p * max_batch + b (the table written above), so both are strided dimensions
     EncodeTiledFn fn = get_encode_fn();
-    const cuuint64_t page_bytes = (cuuint64_t)c->geom.page_elems() * 2;
-    cuuint64_t dims[5] = {64, 16, (cuuint64_t)cfg->n_layers * cfg->n_kv_heads * 4, (cuuint64_t)cfg->max_batch, (cuuint64_t)c->pages_per_seq};
-    cuuint64_t strides[4] = {128, 2048, page_bytes, page_bytes * (cuuint64_t)cfg->max_batch};
-    cuuint32_t box[5] = {64, 16, 1, 1, AU_KT / 16};
+    const cuuint64_t pair_bytes = (cuuint64_t)c->geom.block_elems() * 2 * 2;
+    cuuint64_t dims[5] = {64, 64, (cuuint64_t)cfg->max_batch, (cuuint64_t)c->pages_per_seq, (cuuint64_t)cfg->n_layers * cfg->n_kv_heads};
+    cuuint64_t strides[4] = {128, pair_bytes, pair_bytes * (cuuint64_t)cfg->max_batch, pair_bytes * (cuuint64_t)c->geom.pool_pages()};
+    cuuint32_t box[5] = {64, 16, 1, AU_KT / 16, 1};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     c->tm_kv_ok = fn && fn(&c->tm_kv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, c->d_pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
