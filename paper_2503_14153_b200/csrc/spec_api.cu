@@ -670,10 +670,20 @@ bool attn_rows_mode(const spec_ctx* c, int R) {
   return nw > 1 && c->cfg.n_heads * c->B * nw <= SM_SLOTS / 2;
 }
 
-// Passes of more than 32 rows over a context that may reach long_attn_keys positions.
+// Context length from which a pass of R rows goes to the long-context kernels: the option's value, but at most
+// ATTN_WAVES_KEYS for passes of more than 32 rows whose (sequence, head, 16-row block) CTAs do not fit one wave
+// (batched verification): there the tcgen05 kernel, one CTA per (sequence, head, 64 rows), already wins.
+constexpr int ATTN_WAVES_KEYS = 512;
+int attn_long_threshold(const spec_ctx* c, int R) {
+  const bool umma = c->attn_umma && c->tm_kv_ok && c->cfg.head_dim == 128;
+  if (c->long_attn_keys > 0 && umma && R > 32 && !attn_rows_mode(c, R)) return std::min(c->long_attn_keys, ATTN_WAVES_KEYS);
+  return c->long_attn_keys;
+}
+// Passes of more than 32 rows (any pass with the tcgen05 kernel) over a context that may exceed that length.
 bool attn_long_mode(const spec_ctx* c, int R, int keys_hi) {
   const bool umma = c->attn_umma && c->tm_kv_ok && c->cfg.head_dim == 128;
-  return c->long_attn_keys > 0 && (R > 32 || umma) && keys_hi > c->long_attn_keys;
+  const int thr = attn_long_threshold(c, R);
+  return thr > 0 && (R > 32 || umma) && keys_hi > thr;
 }
 
 // n_hi_pass / n_lo_pass: host bounds of the cached length the pass's rows sit on, per sequence
@@ -1142,8 +1152,8 @@ int step_t(spec_ctx* c, int32_t* out_tokens, int32_t* out_counts, const int32_t*
     // for at most ATTN_SINGLE_TILES tiles or for any length
     int bound;
     if (attn_long_mode(c, T_, c->n_hi[b] + T_)) bound = c->cap;
-    else if (attn_rows_mode(c, T_)) bound = attn_long_mode(c, T_, 1 << 30) ? std::min(c->long_attn_keys / 64 * 64, c->cap) : c->cap;
-    else if (c->n_hi[b] + T_ > ATTN_SINGLE_TILES * 64) bound = attn_long_mode(c, T_, 1 << 30) ? std::min(std::max(c->long_attn_keys / 64 * 64, ATTN_SINGLE_TILES * 64), c->cap) : c->cap;
+    else if (attn_rows_mode(c, T_)) bound = attn_long_mode(c, T_, 1 << 30) ? std::min(attn_long_threshold(c, T_) / 64 * 64, c->cap) : c->cap;
+    else if (c->n_hi[b] + T_ > ATTN_SINGLE_TILES * 64) bound = attn_long_mode(c, T_, 1 << 30) ? std::min(std::max(attn_long_threshold(c, T_) / 64 * 64, ATTN_SINGLE_TILES * 64), c->cap) : c->cap;
     else bound = std::min(ATTN_SINGLE_TILES * 64, c->cap);
     n_hi_plan[b] = bound - T_;
     n_lo_plan[b] = c->n_lo[b];

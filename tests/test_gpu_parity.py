@@ -129,6 +129,32 @@ def test_long_context_attention_kernels_on_small_shapes(torch, T, prompt_len, um
     assert rep.steps > 0
 
 
+@pytest.mark.parametrize("umma", [1, 0])
+def test_long_context_attention_kernels_batched_ragged(torch, umma):
+    """The long-context attention kernels on a batch of four ragged sequences (17 to 530 cached positions: less
+    than one 128-key tile up to several tiles with a ragged tail; sequence b's pages interleave with the others'
+    in the pool), every sequence in lock step with an oracle of its own for three steps."""
+    from oracle.decoder import OracleModel
+    from oracle.spec import OracleSpecDecoder
+    from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights
+    from paper_2503_14153_b200 import binding as B
+    from tests_lockstep import run_lockstep_batch
+    cfg = SMALL_BF16_D128.with_(tree_nodes=64, seed=27)
+    w = draw_weights(cfg)
+    lengths = (17, 530, 129, 256)
+    prompts = [draw_prompt(cfg.with_(seed=27 + i), n) for i, n in enumerate(lengths)]
+    tree = build_tree(cfg.topk, 64)
+    model = OracleModel(cfg, w)
+    gpu = SpecDecoder(cfg, upload_weights(cfg, w), tree, 530 + 40, max_batch=4, flags=B.FLAG_KEEP_LOGITS)
+    gpu.set_option(B.OPT_ATTN_UMMA, umma)
+    gpu.set_option(B.OPT_LONG_ATTN_KEYS, 1)
+    oracles = {b: OracleSpecDecoder(model, tree, 530 + 40) for b in range(4)}
+    reps = run_lockstep_batch(cfg, gpu, oracles, prompts, 3, TOL_BF16, TIE_GAP)
+    gpu.close()
+    for b, rep in reps.items():
+        assert rep.steps == 3, b
+
+
 def test_ten_heads_deep_tree(torch):
     """The paper's head count (K = 10): ten stacked head matrices (three GEMM launches), a tree ten levels deep."""
     cfg = SMALL_BF16.with_(name="small_bf16_k10", n_medusa=10, topk=(4, 3, 2, 2, 2, 1, 1, 1, 1, 1), tree_nodes=48, seed=23)
