@@ -176,19 +176,23 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
  * after a prefill and after an option change; steps that are traced or profiled are enqueued
  * directly). Results do not depend on it. SPEC_OPT_PHASE_TIMING [0]: record an event at the five
  * phase boundaries of every step for spec_last_step_phase_ms (costs the programmatic overlap at
- * those boundaries: about 0.03 ms of a 7B step). SPEC_OPT_CLUSTER_EPILOGUE [2]: bit mask of the projections
+ * those boundaries: about 0.03 ms of a 7B step). SPEC_OPT_CLUSTER_EPILOGUE [6]: bit mask of the projections
  * that, in passes of at most 128 rows, run as thread-block clusters which add their split-K sums through
  * distributed shared memory and apply the step that follows themselves: 1 = output and down projections
  * (residual add in place), 2 = gate+up (SwiGLU, passes of at most 64 rows), 4 = q/k/v (RoPE and cache
  * store). A projection whose bit is clear leaves partial sums for a separate kernel (other summation
- * order, same rounding points). Only bit 2 is on by default: on the 7B shape it is the one that is
- * faster (bits 1 and 4 cost 2% and 4% of a step there). SPEC_OPT_WIDE_GEMM [1]: passes of more than
+ * order, same rounding points). Bits 2 and 4 are on by default: on the 7B shape they shorten a step by 2%
+ * and 4.4% (bit 1 lengthens it by 2%). SPEC_OPT_WIDE_GEMM [1]: passes of more than
  * 128 rows (batched verification, batched prompt processing) run their projections as whole
  * [128 weight rows] x [256 activation rows] tiles that keep a weight tile for 256 rows at a time;
  * 0 = the weight-streaming kernel, which re-reads the weights for every 128 rows.
- * SPEC_OPT_LONG_ATTN_KEYS [2048]: passes of more than 32 rows whose context may exceed this many positions
- * run the attention kernel that shares each K/V tile among the row blocks of a CTA and splits the keys
- * across CTAs (0 = never). Results differ from the other attention kernels only in summation order. */
+ * SPEC_OPT_LONG_ATTN_KEYS [2048]: passes whose context may exceed this many positions run a long-context
+ * attention kernel, in which a CTA reads a head's K/V once for 64 query rows and the keys are split across
+ * the CTAs of a cluster (0 = never; batched passes that need more than one wave of CTAs switch at 512
+ * positions already). SPEC_OPT_ATTN_UMMA [1]: that kernel computes scores and P V on tcgen05 with
+ * accumulators in tensor memory (head_dim 128, 16-row pages); 0 = the mma.sync kernel that shares K/V tiles
+ * between the row blocks of a CTA (passes of more than 32 rows). Results differ from the other attention
+ * kernels only in summation order. */
 enum { SPEC_OPT_PDL = 0, SPEC_OPT_GEMM_CTAS = 1, SPEC_OPT_L2_PREFETCH = 2, SPEC_OPT_TRACE = 3,
        SPEC_OPT_SMALL_GEMM_CTAS = 4, SPEC_OPT_GRAPH = 5, SPEC_OPT_PHASE_TIMING = 6, SPEC_OPT_CLUSTER_EPILOGUE = 7,
        SPEC_OPT_WIDE_GEMM = 8, SPEC_OPT_LONG_ATTN_KEYS = 9,

@@ -14,11 +14,12 @@
 //    2 KC units of the pair are cut into three equal runs, so CTA 0 holds a gate part, CTA 1 a gate
 //    and an up part (two accumulators) and CTA 2 an up part. After the barrier each CTA finishes a
 //    third of the tile's columns: gate = G0 + G1, up = U1 + U2, act = bf16(SiLU(gate) * up).
-//  * GC_ROPE (query, key and value projections, stacked): a cluster of 3 CTAs per 128-row tile of the
-//    stacked matrices, each streaming a third of the K chunks. A tile holds whole heads (head_dim 64 or
+//  * GC_ROPE (query, key and value projections, stacked): a cluster of 2 CTAs per 128-row tile of the
+//    stacked matrices, each streaming half of the K chunks (96 pairs on the 7B shape: all co-resident, which
+//    96 clusters of 3 are not). A tile holds whole heads (head_dim 64 or
 //    128), so after the barrier the cluster rotates the query / key pairs (i, i + head_dim / 2) by the
 //    row's position, writes the bf16 query rows and puts the bf16 key and value rows into the paged cache
-//    at the row's slot; CTA r takes every third activation row.
+//    at the row's slot; CTA r takes every second activation row.
 // Sums are added in a fixed order: results are bit-reproducible. Every wait is bounded; a CTA whose
 // wait ran out still arrives at both cluster barriers, so its cluster mates never wait for it.
 #pragma once
@@ -30,7 +31,7 @@
 namespace spec {
 
 constexpr int GC_RESIDUAL = 0, GC_SWIGLU = 1, GC_ROPE = 2;
-constexpr int GC_RES_CLUSTER = 8, GC_GLU_CLUSTER = 3, GC_ROPE_CLUSTER = 3;
+constexpr int GC_RES_CLUSTER = 8, GC_GLU_CLUSTER = 3, GC_ROPE_CLUSTER = 2;
 
 struct ClusterGemmParams {
   int M, K, KC;                 // activation rows (<= MT), inner size, K / 64
@@ -364,7 +365,7 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
         }
       }
     } else if (MODE == GC_ROPE) {
-      // the tile holds 128 / D whole heads. CTA `rank` takes the activation rows rank, rank + 3, ...; an item is
+      // the tile holds 128 / D whole heads. CTA `rank` takes the activation rows rank, rank + cluster size, ...; an item is
       // (row, group of four rotation pairs): columns [lo, lo + 4) and [lo + D/2, lo + D/2 + 4) of one head
       constexpr int ITEMS = R_ITEMS, PER = R_PER;
       const int half = p.g.head_dim >> 1;
@@ -372,17 +373,20 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
       int (&mrow)[R_PER] = r_mrow, (&lo_c)[R_PER] = r_lo_c;
       float4 (&cs01)[R_PER] = r_cs01, (&cs23)[R_PER] = r_cs23;
       bf16* (&dst)[R_PER] = r_dst;
-      const uint32_t s0 = dsmem_addr(stage_local, 0u), s1 = dsmem_addr(stage_local, 1u), s2 = dsmem_addr(stage_local, 2u);
+      uint32_t sb[CS];
+#pragma unroll
+      for (int r = 0; r < CS; ++r) sb[r] = dsmem_addr(stage_local, (uint32_t)r);
       float4 a[PER], c[PER];
 #pragma unroll
       for (int k = 0; k < PER; ++k) {
         const int lo = lo_c[k] & 0xffff;
         const uint32_t o_lo = (uint32_t)((mrow[k] * Cfg::PITCH + lo) * 4), o_hi = o_lo + (uint32_t)(half * 4);
         const bool ld = (e + 128 * k) < ITEMS && mrow[k] < MT;
-        a[k] = ld ? dsmem_ld4(s0 + o_lo) : make_float4(0.f, 0.f, 0.f, 0.f);
-        c[k] = ld ? dsmem_ld4(s0 + o_hi) : make_float4(0.f, 0.f, 0.f, 0.f);
-        if (ld) { add4(a[k], dsmem_ld4(s1 + o_lo)); add4(c[k], dsmem_ld4(s1 + o_hi)); }
-        if (ld) { add4(a[k], dsmem_ld4(s2 + o_lo)); add4(c[k], dsmem_ld4(s2 + o_hi)); }
+        a[k] = ld ? dsmem_ld4(sb[0] + o_lo) : make_float4(0.f, 0.f, 0.f, 0.f);
+        c[k] = ld ? dsmem_ld4(sb[0] + o_hi) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int r = 1; r < CS; ++r)
+          if (ld) { add4(a[k], dsmem_ld4(sb[r] + o_lo)); add4(c[k], dsmem_ld4(sb[r] + o_hi)); }
       }
 #pragma unroll
       for (int k = 0; k < PER; ++k) {

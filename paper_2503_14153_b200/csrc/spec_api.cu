@@ -207,7 +207,7 @@ struct spec_ctx {
   CUtensorMap tm_kv;                   // 5-D view of the page pool for its TMA loads
   bool tm_kv_ok = false;
   bool wide_gemm = true;               // SPEC_OPT_WIDE_GEMM: passes of more than 128 rows use the 128 x 256-tile kernel
-  int cluster_epilogue = 2;            // SPEC_OPT_CLUSTER_EPILOGUE: which projections finish their split-K sums inside a cluster
+  int cluster_epilogue = 6;            // SPEC_OPT_CLUSTER_EPILOGUE: which projections finish their split-K sums inside a cluster
                                        // (bits: 1 output/down, 2 gate+up, 4 q/k/v; measured on the 7B shape: only gate+up pays)
   int small_gemm_ctas = 288;           // CTAs of GEMMs with at most 48 weight tiles (Wo, down); 288 since the weights are pre-tiled (192 before)
   std::vector<int> h_parent, h_depth, h_rank;
