@@ -35,7 +35,6 @@ constexpr int AU_KT = 128;        // keys per tile
 constexpr int AU_ROWS = 64;       // query rows per CTA
 constexpr int AU_THREADS = 320;   // warps 0..3: softmax group 0; warps 4..7: group 1; warp 8: producer; warp 9: MMA
 constexpr float AU_RESCALE_LOG2 = 8.f;   // a stream's reference is raised when a tile's maximum exceeds it by more than this
-constexpr int AU_SPLIT_TILES = 4; // fewest tiles worth a key split of their own
 constexpr int AU_MAX_CLUSTER = 8; // most key splits (portable cluster size)
 constexpr int AU_EXP = 132;       // floats per staged output row: head_dim + 4 (16-byte aligned rows, banks shifted by 4)
 
@@ -102,10 +101,45 @@ attention_umma(const __grid_constant__ CUtensorMap tm_kv, const AttnTcArgs a, un
   const int h = blockIdx.x, sp = blockIdx.y, b = blockIdx.z / halves, half = blockIdx.z % halves;
   const int row0 = half * AU_ROWS;
   const int H = a.H, kvh = h / (H / a.g.n_kv_heads);
-  if (threadIdx.x == 0) {
+  const int ncl = (int)gridDim.y;                              // key splits = the cluster; split sp owns tiles sp, sp + ncl, ...
+  // ---- producer's loads: two K slabs and two V slabs per tile, K one tile ahead of V (K is released by the
+  // score MMAs, long before the tile's V is released by the P V MMAs) ----
+  const int lh = a.layer * a.g.n_kv_heads + kvh;             // slab rows of a page's pair: K dims 0..63, K 64..127, V, V
+  auto load_k = [&](int t) -> bool {
+    const int st = t & 1;
+    if (t >= 2 && !mbar_wait(&k_empty[st], ((t >> 1) - 1) & 1, a.status, 50)) return false;
+    uint8_t* dst = kv_s + st * 65536;
+    mbar_expect_tx(&k_full[st], 32768);
+    const int page0 = (sp + t * ncl) * (AU_KT / 16);
+    tma_load_5d(dst, &tm_kv, 0, 0, b, page0, lh, &k_full[st]);
+    tma_load_5d(dst + 16384, &tm_kv, 0, 16, b, page0, lh, &k_full[st]);
+    return true;
+  };
+  auto load_v = [&](int t) -> bool {
+    const int st = t & 1;
+    if (t >= 2 && !mbar_wait(&v_empty[st], ((t >> 1) - 1) & 1, a.status, 56)) return false;
+    uint8_t* dst = kv_s + st * 65536 + 32768;
+    mbar_expect_tx(&v_full[st], 32768);
+    const int page0 = (sp + t * ncl) * (AU_KT / 16);
+    tma_load_5d(dst, &tm_kv, 0, 32, b, page0, lh, &v_full[st]);
+    tma_load_5d(dst + 16384, &tm_kv, 0, 48, b, page0, lh, &v_full[st]);
+    return true;
+  };
+  // The producer thread sets up the barriers itself and at once asks for its first two tiles where they lie
+  // wholly below the host's lower bound of the committed length: those keys were written by earlier steps (no
+  // kernel of this step starts before the kernels of the step before it have completed), so the loads need not
+  // wait for the kernel before this one, and which tiles a split owns does not depend on the length.
+  int pre = 0;                                                 // tiles whose loads went out before the dependency wait
+  if (threadIdx.x == 8 * 32) {
     for (int i = 0; i < 14; ++i) mbar_init(&bars[i], (i == 10 || i == 11) ? 4 : 1);
     mbar_fence_init();
-    tma_prefetch_desc(&tm_kv);
+    const int n_lo = b < ATTN_MAX_SEQS ? a.n_lo[b] : 0;
+    if ((sp + 1) * AU_KT <= n_lo) {
+      load_k(0);
+      pre = 1;
+      if ((sp + ncl + 1) * AU_KT <= n_lo) { load_k(1); pre = 2; }
+      load_v(0);
+    }
   }
   if (warp == 9) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
   // the P operands' off-diagonal blocks stay zero for the whole kernel
@@ -122,46 +156,40 @@ attention_umma(const __grid_constant__ CUtensorMap tm_kv, const AttnTcArgs a, un
   const int R = a.rows.R, cnt = a.rows.cnt[b], n = a.rows.n[b];
   const int S = n + cnt;
   const int total_tiles = (S + AU_KT - 1) / AU_KT;
-  const int nsplit = max(1, min(a.nsplit, (total_tiles + AU_SPLIT_TILES - 1) / AU_SPLIT_TILES));
-  const int tps = (total_tiles + nsplit - 1) / nsplit;
-  const int t0 = sp * tps, nt = min(total_tiles, t0 + tps) - t0;
-  const bool active = row0 < cnt && sp < nsplit && nt > 0;
-  // ---- producer's loads: two K slabs and two V slabs per tile, K one tile ahead of V (K is released by the
-  // score MMAs, long before the tile's V is released by the P V MMAs) ----
-  const int lh = a.layer * a.g.n_kv_heads + kvh;             // slab rows of a page's pair: K dims 0..63, K 64..127, V, V
-  auto load_k = [&](int t) -> bool {
-    const int st = t & 1;
-    if (t >= 2 && !mbar_wait(&k_empty[st], ((t >> 1) - 1) & 1, a.status, 50)) return false;
-    uint8_t* dst = kv_s + st * 65536;
-    mbar_expect_tx(&k_full[st], 32768);
-    const int page0 = (t0 + t) * (AU_KT / 16);
-    tma_load_5d(dst, &tm_kv, 0, 0, b, page0, lh, &k_full[st]);
-    tma_load_5d(dst + 16384, &tm_kv, 0, 16, b, page0, lh, &k_full[st]);
-    return true;
-  };
-  auto load_v = [&](int t) -> bool {
-    const int st = t & 1;
-    if (t >= 2 && !mbar_wait(&v_empty[st], ((t >> 1) - 1) & 1, a.status, 56)) return false;
-    uint8_t* dst = kv_s + st * 65536 + 32768;
-    mbar_expect_tx(&v_full[st], 32768);
-    const int page0 = (t0 + t) * (AU_KT / 16);
-    tma_load_5d(dst, &tm_kv, 0, 32, b, page0, lh, &v_full[st]);
-    tma_load_5d(dst + 16384, &tm_kv, 0, 48, b, page0, lh, &v_full[st]);
-    return true;
-  };
+  const int nt = sp < total_tiles ? (total_tiles - sp + ncl - 1) / ncl : 0;   // (pre <= nt: the tiles asked for lie below n)
+  const bool active = row0 < cnt && nt > 0;
   if (active) {
     if (warp == 8) {
       // the first tiles are on their way while the other warps stage Q
-      if (lane == 0) { load_k(0); if (nt > 1) load_k(1); load_v(0); }
+      if (lane == 0) {
+        if (pre < 1) load_k(0);
+        if (pre < 2 && nt > 1) load_k(1);
+        if (pre < 1) load_v(0);
+      }
     } else if (warp < 8) {
-      // Q rows of this CTA, twice, into the two K-major slabs (rows beyond cnt are zeros)
-      for (int c = threadIdx.x; c < 2 * AU_ROWS * (HD / 8); c += 256) {
-        const int r = c / (HD / 8), ch = c % (HD / 8), qr = r & (AU_ROWS - 1);
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (row0 + qr < cnt) v = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + row0 + qr) * H * HD + h * HD + ch * 8);
-        *reinterpret_cast<uint4*>(q_s + (ch >> 3) * 16384 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = v;
+      // Q rows of this CTA into the two K-major slabs, each row at r and at r + 64 (rows beyond cnt are zeros);
+      // a thread fetches its four pieces before it stores the first
+      uint4 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int c = threadIdx.x + 256 * k, qr = c / (HD / 8), ch = c % (HD / 8);
+        v[k] = make_uint4(0, 0, 0, 0);
+        if (row0 + qr < cnt) v[k] = *reinterpret_cast<const uint4*>(a.q + (size_t)(b * R + row0 + qr) * H * HD + h * HD + ch * 8);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int c = threadIdx.x + 256 * k, qr = c / (HD / 8), ch = c % (HD / 8);
+        uint8_t* dst = q_s + (ch >> 3) * 16384 + qr * 128 + (((ch & 7) ^ (qr & 7)) << 4);   // (qr + 64) & 7 == qr & 7
+        *reinterpret_cast<uint4*>(dst) = v[k];
+        *reinterpret_cast<uint4*>(dst + AU_ROWS * 128) = v[k];
       }
     }
+  } else if (pre > 0 && threadIdx.x == 8 * 32) {
+    // rows beyond the pass's count: nothing to do, but the loads asked for above must have landed before the
+    // CTA gives up its shared memory
+    mbar_wait(&k_full[0], 0, a.status, 59);
+    mbar_wait(&v_full[0], 0, a.status, 59);
+    if (pre > 1) mbar_wait(&k_full[1], 0, a.status, 59);
   }
   fence_proxy_async_smem();
   __syncthreads();
@@ -242,7 +270,7 @@ attention_umma(const __grid_constant__ CUtensorMap tm_kv, const AttnTcArgs a, un
         if (!mbar_wait(&s_full[bf], (t >> 1) & 1, a.status, 54)) { ok = false; break; }
         tc_fence_after();
         const uint32_t s_addr = tmem + lane_base + (uint32_t)(bf * 128 + kh * 64);
-        const int k0 = (t0 + t) * AU_KT + kh * 64;             // first key of this thread's half
+        const int k0 = (sp + t * ncl) * AU_KT + kh * 64;       // first key of this thread's half
         uint32_t r0[32], r1[32];
         tmem_ld32(s_addr, r0);
         tmem_ld32(s_addr + 32, r1);
@@ -360,7 +388,6 @@ attention_umma(const __grid_constant__ CUtensorMap tm_kv, const AttnTcArgs a, un
   }
   __syncthreads();
   if (warp == 9) { tc_fence_after(); tmem_dealloc(tmem, 512); }
-  const int ncl = (int)gridDim.y;                              // cluster = the key splits of this (sequence, row half, head)
   if (warp < 8) {
     // thread = (row, every fourth 4-dim chunk): merge the four streams
     const int row = threadIdx.x >> 2, qd = threadIdx.x & 3;

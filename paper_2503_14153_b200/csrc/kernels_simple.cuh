@@ -17,8 +17,12 @@ __global__ void prepare_verify_rows(Rows rows, const int* __restrict__ cand, int
                                     const T* __restrict__ embed, float* __restrict__ x, int d, int vocab,
                                     int* status, unsigned long long* tr) {
   KTrace kt(tr);
-  pdl_launch_dependents();
+  // This kernel lets its dependents start only after its own dependency wait, i.e. after every kernel before it
+  // has completed: no kernel of the verification pass begins before the previous step's kernels (its cache
+  // compaction above all) are done. The attention kernels rely on that when they fetch keys below the host's
+  // lower bound of the committed length ahead of their own dependency wait.
   pdl_wait();
+  pdl_launch_dependents();
   if (threadIdx.x == 0) trace_mark_min(tr, 2);
   int m = blockIdx.x, b = m / rows.R, i = m % rows.R;
   int n = rows.n[b];
