@@ -12,8 +12,10 @@
 //    follows needs the row's mean square) in ss_part[m][tile * 8 + r].
 //  * GC_SWIGLU (gate and up projections): a cluster of 3 CTAs per pair (gate tile t, up tile t); the
 //    2 KC units of the pair are cut into three equal runs, so CTA 0 holds a gate part, CTA 1 a gate
-//    and an up part (two accumulators) and CTA 2 an up part. After the barrier each CTA finishes a
-//    third of the tile's columns: gate = G0 + G1, up = U1 + U2, act = bf16(SiLU(gate) * up).
+//    and an up part (two accumulators) and CTA 2 an up part. Once every CTA's MMAs are complete (first
+//    barrier) each thread sends the values of its weight row into the shared memory of the CTA that finishes
+//    that column (remote stores); after the second barrier each CTA finishes a third of the tile's columns
+//    from its own shared memory: gate = G0 + G1, up = U1 + U2, act = bf16(SiLU(gate) * up).
 //  * GC_ROPE (query, key and value projections, stacked): a cluster of 2 CTAs per 128-row tile of the
 //    stacked matrices, each streaming half of the K chunks (96 pairs on the 7B shape: all co-resident, which
 //    96 clusters of 3 are not). A tile holds whole heads (head_dim 64 or
@@ -83,6 +85,9 @@ __device__ __forceinline__ float4 dsmem_ld4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
   return v;
+}
+__device__ __forceinline__ void dsmem_st(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 __device__ __forceinline__ void add4(float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
 
@@ -282,7 +287,10 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
     const int q = warp & 3;
     pdl_wait();
     if (MODE == GC_ROPE) rope_meta();
-    if (n_units > 0 && mbar_wait(acc_full, 0, p.status, 32)) {
+    if (MODE == GC_SWIGLU) {
+      // the accumulators stay in tensor memory until every CTA of the cluster has finished its MMAs (below)
+      if (n_units > 0) mbar_wait(acc_full, 0, p.status, 32);
+    } else if (n_units > 0 && mbar_wait(acc_full, 0, p.status, 32)) {
       tc_fence_after();
       for (int s = 0; s < nseg; ++s) {
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(s * MT);
@@ -309,9 +317,78 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
     }
   }
 
-  // ---- every thread of every CTA of the cluster: the staged accumulators are complete ----
+  // ---- every thread of every CTA of the cluster: the staged accumulators are complete (GC_SWIGLU: every CTA's
+  // MMAs are complete, so every ring is free) ----
   __syncwarp();
   cluster_sync_all();
+
+  if (MODE == GC_SWIGLU) {
+    // Push instead of pull: a thread owns weight row w of its CTA's accumulators and sends its MT values
+    // straight into the shared memory of the CTA that finishes column w (rows 0..43 -> CTA 0, 44..83 -> CTA 1,
+    // 84..127 -> CTA 2) with remote stores, which nobody waits for; after the next barrier each CTA reads only
+    // its own shared memory. Four compact buffers [MT][GLU_PITCH] per CTA: gate parts of CTA 0 and CTA 1, up
+    // parts of CTA 1 and CTA 2. (Reading the parts through distributed shared memory instead took 4.4 us.)
+    constexpr int CP = 48;                                    // floats per staged row (44 columns at most)
+    static_assert(4 * MT * CP * 4 <= Cfg::RING_BYTES, "four compact buffers must fit the ring");
+    if (warp >= 2 && n_units > 0) {
+      const int q = warp & 3, w = q * 32 + lane;
+      const int own = w < 44 ? 0 : (w < 84 ? 1 : 2);
+      const int col = w - (own == 0 ? 0 : (own == 1 ? 44 : 84));
+      const uint32_t dst0 = dsmem_addr(smem_u32(staging), (uint32_t)own);
+      tc_fence_after();
+      for (int s2 = 0; s2 < nseg; ++s2) {
+        const int slot = seg[s2].mat == 0 ? rank : rank + 1;
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(s2 * MT);
+        const uint32_t dst = dst0 + (uint32_t)((slot * MT * CP + col) * 4);
+        if (MT >= 32) {
+#pragma unroll
+          for (int g = 0; g < MT / 32; ++g) {
+            uint32_t r[32];
+            tmem_ld32(taddr + g * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) dsmem_st(dst + (uint32_t)((g * 32 + j) * CP * 4), __uint_as_float(r[j]));
+          }
+        } else {
+          uint32_t r[16];
+          tmem_ld16(taddr, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) dsmem_st(dst + (uint32_t)(j * CP * 4), __uint_as_float(r[j]));
+        }
+      }
+      tc_fence_before();
+    }
+    __syncwarp();
+    cluster_sync_all();                                       // the parts have arrived (release / acquire)
+    if (warp >= 2 && n_units > 0) {
+      const int e = threadIdx.x - 64;
+      const int lo = rank == 0 ? 0 : (rank == 1 ? 44 : 84), hi = rank == 0 ? 44 : (rank == 1 ? 84 : 128);
+      const int gpr = (hi - lo) >> 2;                        // groups of four columns per row: 11, 10, 11
+      constexpr int PER = (MT * 11 + 127) / 128;
+      const float* b0 = staging;
+#pragma unroll
+      for (int k = 0; k < PER; ++k) {
+        const int it = e + 128 * k, m = it / gpr, w4 = it % gpr;
+        const int col = t * 128 + lo + 4 * w4;
+        if (m < MT && m < p.M && col < p.N) {
+          const float* src = b0 + m * CP + 4 * w4;
+          float4 ga = *reinterpret_cast<const float4*>(src), ua = *reinterpret_cast<const float4*>(src + 2 * MT * CP);
+          add4(ga, *reinterpret_cast<const float4*>(src + MT * CP));
+          add4(ua, *reinterpret_cast<const float4*>(src + 3 * MT * CP));
+          uint2 o;
+          o.x = pack_bf16x2(silu_f(ga.x) * ua.x, silu_f(ga.y) * ua.y);
+          o.y = pack_bf16x2(silu_f(ga.z) * ua.z, silu_f(ga.w) * ua.w);
+          *reinterpret_cast<uint2*>(p.act + (size_t)m * p.N + col) = o;
+        }
+      }
+    }
+    // nobody writes to or reads from another CTA's shared memory after the second barrier: no third one
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+    return;
+  }
 
   if (warp >= 2 && n_units > 0) {
     // Every finishing thread issues all its loads (distributed shared memory, residual stream) before it
@@ -405,36 +482,6 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
         const int up = rope_mat == 0 ? half : (lo_c[k] >> 16);
         *reinterpret_cast<uint2*>(dst[k]) = lo_o;
         *reinterpret_cast<uint2*>(dst[k] + up) = hi_o;
-      }
-    } else {
-      // CTA `rank` finishes weight rows [lo, hi) of the pair for every activation row: gate parts sit in CTA 0
-      // (buffer 0) and CTA 1 (buffer 0), up parts in CTA 1 (buffer 1) and CTA 2 (buffer 0); an item is
-      // (row m, group of four output columns)
-      const int lo = rank == 0 ? 0 : (rank == 1 ? 44 : 84), hi = rank == 0 ? 44 : (rank == 1 ? 84 : 128);
-      const int gpr = (hi - lo) >> 2;                        // groups per row: 11, 10, 11
-      constexpr int PER = (MT * 11 + 127) / 128;
-      const uint32_t g0 = dsmem_addr(stage_local, 0u), g1 = dsmem_addr(stage_local, 1u);
-      const uint32_t u1 = g1 + (uint32_t)(Cfg::STAGING_FLOATS * 4), u2 = dsmem_addr(stage_local, 2u);
-      float4 ga[PER], ua[PER];
-#pragma unroll
-      for (int k = 0; k < PER; ++k) {
-        const int it = e + 128 * k, m = it / gpr, w4 = it % gpr;
-        const bool ld = m < MT;
-        const uint32_t off = (uint32_t)((m * Cfg::PITCH + lo + 4 * w4) * 4);
-        ga[k] = ld ? dsmem_ld4(g0 + off) : make_float4(0.f, 0.f, 0.f, 0.f);
-        ua[k] = ld ? dsmem_ld4(u1 + off) : make_float4(0.f, 0.f, 0.f, 0.f);
-        if (ld) { add4(ga[k], dsmem_ld4(g1 + off)); add4(ua[k], dsmem_ld4(u2 + off)); }
-      }
-#pragma unroll
-      for (int k = 0; k < PER; ++k) {
-        const int it = e + 128 * k, m = it / gpr, w4 = it % gpr;
-        const int col = t * 128 + lo + 4 * w4;
-        if (m < MT && m < p.M && col < p.N) {
-          uint2 o;
-          o.x = pack_bf16x2(silu_f(ga[k].x) * ua[k].x, silu_f(ga[k].y) * ua[k].y);
-          o.y = pack_bf16x2(silu_f(ga[k].z) * ua[k].z, silu_f(ga[k].w) * ua[k].w);
-          *reinterpret_cast<uint2*>(p.act + (size_t)m * p.N + col) = o;
-        }
       }
     }
   }
