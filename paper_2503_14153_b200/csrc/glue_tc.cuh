@@ -19,6 +19,7 @@ struct PartView {
   int ld;
   SegMap seg;                  // how the GEMM dealt its units: gives the slots of a tile
   int mt_shift;                // log2 of the activation rows per tile
+  int single;                  // 1: every tile is one finished slot (the 128 x 256-tile GEMM): read it directly
 };
 
 constexpr int PV_UNROLL = 12;
@@ -40,6 +41,11 @@ __device__ __forceinline__ float4 part_sum4(const PartView& pv, int m, int colp)
     a.x += w.x; a.y += w.y; a.z += w.z; a.w += w.w;
   }
   return a;
+}
+
+// The same for a view of finished sums (pv.single).
+__device__ __forceinline__ float4 part_one4(const PartView& pv, int m, int colp) {
+  return __ldcg(reinterpret_cast<const float4*>(pv.part + (size_t)m * pv.ld + colp));
 }
 
 __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
@@ -145,6 +151,89 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
     emit(c4, *reinterpret_cast<const float4*>(xr + c4 * 4), *reinterpret_cast<const float4*>(gain + c4 * 4));
 }
 
+// The same operation for passes of many rows (batched verification, prompt processing): one CTA of
+// NORMW_THREADS per row, no cluster. With hundreds of rows the kernel is bound by bandwidth, not by the
+// latency of one row, so what counts is loads in flight: a thread fetches all its pieces of x and of the
+// partial sums before it uses the first (NORMW_CACHE float4 each; rows longer than that loop).
+constexpr int NORMW_THREADS = 256;
+constexpr int NORMW_CACHE = 4;
+
+__global__ void __launch_bounds__(NORMW_THREADS)
+norm_rows_wide(float* __restrict__ x, const PartView pv, const float* __restrict__ gain, float eps,
+               bf16* __restrict__ u, float* __restrict__ hid, int d, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  const int m = blockIdx.x;
+  float* xr = x + (size_t)m * d;
+  const int n4 = d >> 2;
+  float4 gk[NORMW_CACHE];
+#pragma unroll
+  for (int k = 0; k < NORMW_CACHE; ++k) {
+    const int c4 = threadIdx.x + k * NORMW_THREADS;
+    gk[k] = c4 < n4 ? *reinterpret_cast<const float4*>(gain + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  auto part4 = [&](int c4) { return pv.single ? part_one4(pv, m, c4 * 4) : part_sum4(pv, m, c4 * 4); };
+  float4 keep[NORMW_CACHE], add[NORMW_CACHE];
+#pragma unroll
+  for (int k = 0; k < NORMW_CACHE; ++k) {
+    const int c4 = threadIdx.x + k * NORMW_THREADS;
+    keep[k] = add[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c4 < n4) {
+      keep[k] = *reinterpret_cast<const float4*>(xr + c4 * 4);
+      if (pv.part) add[k] = part4(c4);
+    }
+  }
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < NORMW_CACHE; ++k) {
+    const int c4 = threadIdx.x + k * NORMW_THREADS;
+    if (c4 < n4) {
+      float4& v = keep[k];
+      if (pv.part) {
+        v.x += add[k].x; v.y += add[k].y; v.z += add[k].z; v.w += add[k].w;
+        *reinterpret_cast<float4*>(xr + c4 * 4) = v;
+      }
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+  }
+  for (int c4 = threadIdx.x + NORMW_CACHE * NORMW_THREADS; c4 < n4; c4 += NORMW_THREADS) {
+    float4 v = *reinterpret_cast<const float4*>(xr + c4 * 4);
+    if (pv.part) {
+      const float4 a = part4(c4);
+      v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+      *reinterpret_cast<float4*>(xr + c4 * 4) = v;
+    }
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  __shared__ float red[NORMW_THREADS / 32];
+  __shared__ float row_ss;
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < NORMW_THREADS / 32; ++w) t += red[w];
+    row_ss = t;
+  }
+  __syncthreads();
+  const float inv = rsqrtf(row_ss / (float)d + eps);
+  auto emit = [&](int c4, const float4& v, const float4& g) {
+    const float4 o = make_float4(v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
+    *reinterpret_cast<uint2*>(u + (size_t)m * d + c4 * 4) = pack4_bf16(o.x, o.y, o.z, o.w);
+    if (hid) *reinterpret_cast<float4*>(hid + (size_t)m * d + c4 * 4) = o;
+  };
+#pragma unroll
+  for (int k = 0; k < NORMW_CACHE; ++k) {
+    const int c4 = threadIdx.x + k * NORMW_THREADS;
+    if (c4 < n4) emit(c4, keep[k], gk[k]);
+  }
+  for (int c4 = threadIdx.x + NORMW_CACHE * NORMW_THREADS; c4 < n4; c4 += NORMW_THREADS)
+    emit(c4, *reinterpret_cast<const float4*>(xr + c4 * 4), *reinterpret_cast<const float4*>(gain + c4 * 4));
+}
+
 // ------------------------------------------------------------------ RoPE + cache store
 // Sums the QKV partial slots, rotates q and k (rotate-half pairs (e, e + D/2), table
 // cs[pos][e] = (cos, sin)), writes q as bf16 [M][H*D] and k, v as bf16 into the paged cache at
@@ -165,12 +254,19 @@ rope_store_tc(const PartView pv, int qp0, int kp0, int vp0, Rows rows, const flo
   const int tid = blockIdx.y * blockDim.x + threadIdx.x, nthr = gridDim.y * blockDim.x;
   // row bookkeeping and partial sums are independent loads: issue them together
   const int cnt = rows.cnt[b], pos = rows.pos[m], slot = rows.slot[m];
-  for (int it = tid; it < n_rot + n_v; it += nthr) {
+  // item -> first padded column of its group of four (rotated items also take the group half a head further)
+  auto item_col = [&](int it) {
     if (it < n_rot) {
       const int head = it / q4, e = (it % q4) * 4;
-      const int colp = (head < H ? qp0 + head * D : kp0 + (head - H) * D) + e;
-      const float4 a = part_sum4(pv, m, colp), c = part_sum4(pv, m, colp + half);
-      if (i >= cnt) continue;
+      return (head < H ? qp0 + head * D : kp0 + (head - H) * D) + e;
+    }
+    const int iv = it - n_rot;
+    return vp0 + (iv / (D >> 2)) * D + (iv % (D >> 2)) * 4;
+  };
+  auto finish = [&](int it, const float4& a, const float4& c) {
+    if (i >= cnt) return;
+    if (it < n_rot) {
+      const int head = it / q4, e = (it % q4) * 4;
       const float4 t01 = *reinterpret_cast<const float4*>(cs + (size_t)pos * half + e);
       const float4 t23 = *reinterpret_cast<const float4*>(cs + (size_t)pos * half + e + 2);
       const uint2 lo = pack4_bf16(a.x * t01.x - c.x * t01.y, a.y * t01.z - c.y * t01.w, a.z * t23.x - c.z * t23.y, a.w * t23.z - c.w * t23.w);
@@ -188,12 +284,39 @@ rope_store_tc(const PartView pv, int qp0, int kp0, int vp0, Rows rows, const flo
     } else {
       const int iv = it - n_rot;
       const int kh = iv / (D >> 2), e = (iv % (D >> 2)) * 4;
-      const float4 a = part_sum4(pv, m, vp0 + kh * D + e);
-      if (i >= cnt) continue;
       const int page = page_table[b * g.pages_per_seq + slot / g.page_size], prow = slot % g.page_size;
       bf16* dst = pool + g.block_offset(page, layer, 1, kh) + (size_t)prow * D;
       *reinterpret_cast<uint2*>(dst + kv_elem<bf16>(prow, e, D, g.page_size)) = pack4_bf16(a.x, a.y, a.z, a.w);
     }
+  };
+  if (pv.single) {
+    // passes of many rows (finished sums): a thread keeps the loads of four items in flight
+    constexpr int U = 4;
+    for (int it0 = tid; it0 < n_rot + n_v; it0 += U * nthr) {
+      float4 a[U], c[U];
+#pragma unroll
+      for (int k = 0; k < U; ++k) {
+        const int it = it0 + k * nthr;
+        a[k] = c[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (it < n_rot + n_v) {
+          const int colp = item_col(it);
+          a[k] = part_one4(pv, m, colp);
+          if (it < n_rot) c[k] = part_one4(pv, m, colp + half);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < U; ++k) {
+        const int it = it0 + k * nthr;
+        if (it < n_rot + n_v) finish(it, a[k], c[k]);
+      }
+    }
+    return;
+  }
+  for (int it = tid; it < n_rot + n_v; it += nthr) {
+    const int colp = item_col(it);
+    const float4 a = part_sum4(pv, m, colp);
+    const float4 c = it < n_rot ? part_sum4(pv, m, colp + half) : make_float4(0.f, 0.f, 0.f, 0.f);
+    finish(it, a, c);
   }
 }
 
@@ -208,6 +331,34 @@ swiglu_reduce_tc(const PartView pv, int gp0, int up0, bf16* __restrict__ act, in
   if (threadIdx.x == 0) trace_mark_min(tr, 2);
   const int f4 = F >> 2;
   const size_t total = (size_t)M * f4;
+  if (pv.single) {
+    // passes of many rows (finished sums, hundreds of MB): bandwidth-bound, so a thread keeps the loads of four
+    // items in flight
+    constexpr int U = 4;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t idx0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx0 < total; idx0 += U * stride) {
+      float4 gt[U], up[U];
+#pragma unroll
+      for (int k = 0; k < U; ++k) {
+        const size_t idx = idx0 + k * stride;
+        if (idx < total) {
+          const int m = (int)(idx / f4), f = (int)(idx % f4) * 4;
+          gt[k] = part_one4(pv, m, gp0 + f);
+          up[k] = part_one4(pv, m, up0 + f);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < U; ++k) {
+        const size_t idx = idx0 + k * stride;
+        if (idx < total) {
+          const int m = (int)(idx / f4), f = (int)(idx % f4) * 4;
+          *reinterpret_cast<uint2*>(act + (size_t)m * F + f) =
+              pack4_bf16(silu_f(gt[k].x) * up[k].x, silu_f(gt[k].y) * up[k].y, silu_f(gt[k].z) * up[k].z, silu_f(gt[k].w) * up[k].w);
+        }
+      }
+    }
+    return;
+  }
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
     const int m = (int)(idx / f4), f = (int)(idx % f4) * 4;
     const float4 gt = part_sum4(pv, m, gp0 + f), up = part_sum4(pv, m, up0 + f);

@@ -521,6 +521,7 @@ int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* c
     v.part = c->d_part; v.slot_stride = (size_t)M * tiles_all * 128; v.ld = tiles_all * 128;
     v.seg.KC = w.KC; v.seg.m_tiles = w.m_tiles; v.seg.G = w.n_tiles * w.m_tiles; v.seg.total = (int)total;
     v.mt_shift = 8;
+    v.single = 1;
     *view = v;
     return SPEC_OK;
   }
@@ -809,8 +810,13 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, cons
   bf16* act = static_cast<bf16*>(c->d_act);
   const int kp0 = (HD + 127) / 128 * 128, vp0 = kp0 + (KD + 127) / 128 * 128;   // padded columns of k and v in the QKV partials
   const int up0 = (F + 127) / 128 * 128;                                        // and of the up projection
+  // (passes of more than 128 rows are bound by bandwidth, not by a row's latency: one plain CTA per row)
 #define NORM_LAUNCH(pv, gain, uq, hid)                                                                   \
-  KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M, NORM_CLUSTER), dim3(NORM_THREADS), 0, c->d_x, pv, gain, f.rms_eps, uq, hid, d)
+  if (M > 128) {                                                                                         \
+    KLAUNCH("norm_reduce_tc", norm_rows_wide, dim3(M), dim3(NORMW_THREADS), 0, c->d_x, pv, gain, f.rms_eps, uq, hid, d); \
+  } else {                                                                                               \
+    KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M, NORM_CLUSTER), dim3(NORM_THREADS), 0, c->d_x, pv, gain, f.rms_eps, uq, hid, d); \
+  }
   PartView pend{};              // partial sums of the previous down-projection still to be added to x
   for (int l = 0; l < f.n_layers; ++l) {
     NORM_LAUNCH(pend, c->an[l], u, (float*)nullptr);
@@ -824,7 +830,7 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, cons
       } else {
         PartView vq{};
         if ((r = run_gemm(c, u, M, d, 3, mats, rws, SPEC_PROFILE_QKV, &vq))) return r;
-        KLAUNCH("rope_store_tc", rope_store_tc, dim3(M, M <= 128 ? 8 : 1), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope,
+        KLAUNCH("rope_store_tc", rope_store_tc, dim3(M, M <= 128 ? 8 : 2), dim3(256), 0, vq, 0, kp0, vp0, rows, c->d_rope,
                 static_cast<bf16*>(c->d_q), static_cast<bf16*>(c->d_pool), c->geom, c->d_page_table, l, H);
       }
     }
