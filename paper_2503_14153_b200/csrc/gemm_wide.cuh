@@ -12,7 +12,9 @@
 // tile run side by side and the weights cross HBM once.
 //
 // Warp roles: warp 0 feeds a ring of 48 KB stages (16 KB weight unit by bulk copy or TMA, 32 KB activation
-// tile by TMA, 128-byte swizzle), warp 1 issues tcgen05.mma (M 128, N 256, K 16), warps 2..5 drain.
+// tile by TMA, 128-byte swizzle), warp 1 issues tcgen05.mma (M 128, N 256, K 16), warps 2..9 drain: two warps
+// per SM quarter, one for each half of the tile's 256 activation rows, so that the drain of the last tile (which
+// nothing hides) takes half as long.
 #pragma once
 #include <cuda.h>
 
@@ -44,7 +46,9 @@ struct WideCfg {
   static constexpr int TMEM_COLS = 2 * GW_NT;
 };
 
-__global__ void __launch_bounds__(192, 1)
+constexpr int GW_THREADS = 320;
+
+__global__ void __launch_bounds__(GW_THREADS, 1)
 gemm_wide(const __grid_constant__ StreamTmaps tm, const WideGemmParams p) {
   using Cfg = WideCfg;
   constexpr int STAGES = GW_STAGES;
@@ -69,7 +73,7 @@ gemm_wide(const __grid_constant__ StreamTmaps tm, const WideGemmParams p) {
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(&acc_full[0], 1); mbar_init(&acc_full[1], 1);
-    mbar_init(&acc_empty[0], 4); mbar_init(&acc_empty[1], 4);
+    mbar_init(&acc_empty[0], 8); mbar_init(&acc_empty[1], 8);
     mbar_fence_init();
     for (int i = 0; i < p.n_mats; ++i) if (!p.packed[i]) tma_prefetch_desc(&tm.a[i]);
     tma_prefetch_desc(&tm.b);
@@ -161,8 +165,9 @@ gemm_wide(const __grid_constant__ StreamTmaps tm, const WideGemmParams p) {
       trace_mark_max(p.trace, 3);
     }
   } else {
-    // ---- epilogue: warps 2..5; warp w may touch tensor-memory lanes [32 (w % 4), +32) ----
-    const int q = warp & 3;
+    // ---- epilogue: warps 2..9; warp w may touch tensor-memory lanes [32 (w % 4), +32); warps 2..5 take
+    // activation rows [0, 128) of the tile, warps 6..9 rows [128, 256) ----
+    const int q = warp & 3, hf = warp >= 6 ? 1 : 0;
     pdl_wait();
     const size_t ld = (size_t)p.n_tiles * 128;
     for (int i = 0; i < my_tiles; ++i) {
@@ -175,7 +180,7 @@ gemm_wide(const __grid_constant__ StreamTmaps tm, const WideGemmParams p) {
       float* dst = p.part + (size_t)nt * 128 + q * 32 + lane;
       const int m0 = mt * GW_NT;
 #pragma unroll 2
-      for (int g = 0; g < GW_NT / 32; ++g) {
+      for (int g = hf * (GW_NT / 64); g < (hf + 1) * (GW_NT / 64); ++g) {
         uint32_t r[32];
         tmem_ld32(taddr + g * 32, r);
         tmem_ld_wait();

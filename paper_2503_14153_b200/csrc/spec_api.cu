@@ -512,7 +512,7 @@ int run_gemm(spec_ctx* c, const void* x, int M, int K, int n_mats, const void* c
       static bool set_dev[kAttrDevices] = {};
       bool& set_ = *attr_flag(set_dev);
       if (!set_) { CUDA_OK(cudaFuncSetAttribute(gemm_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, WideCfg::SMEM_BYTES)); set_ = true; }
-      cudaError_t e = launch_k(c->pdl, gemm_wide, dim3(grid), dim3(192), (size_t)WideCfg::SMEM_BYTES, c->stream, tmw, w);
+      cudaError_t e = launch_k(c->pdl, gemm_wide, dim3(grid), dim3(GW_THREADS), (size_t)WideCfg::SMEM_BYTES, c->stream, tmw, w);
       c->launches++;
       if (e != cudaSuccess) return c->fail(SPEC_E_CUDA, std::string("gemm_wide launch: ") + cudaGetErrorString(e));
     }
