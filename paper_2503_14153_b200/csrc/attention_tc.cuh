@@ -60,6 +60,7 @@ struct AttnTcArgs {
   int stages;           // KV tiles in flight per CTA (2..ATTN_MAX_STAGES, at least KG); sizes the shared memory
   int n_lo[ATTN_MAX_SEQS];   // host's lower bound of each sequence's committed length: keys below it
                              // were written by earlier steps and may be fetched before the dependency wait
+  unsigned char order[ATTN_MAX_SEQS];   // attention_umma: sequence taken by the z-th group of CTAs, longest first
   float scale_log2;     // log2(e) / sqrt(head_dim)
   bf16* out;            // [M][H*HD]
   unsigned int* arrive; // [B][H] arrival counters, zero between launches

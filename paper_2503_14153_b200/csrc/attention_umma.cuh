@@ -98,7 +98,10 @@ attention_umma(const __grid_constant__ CUtensorMap tm_kv, const AttnTcArgs a, un
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int halves = gridDim.z / a.rows.B;
-  const int h = blockIdx.x, sp = blockIdx.y, b = blockIdx.z / halves, half = blockIdx.z % halves;
+  // CTAs are handed out in grid order: with more CTAs than SMs the longest sequences go first, so that the
+  // launch does not end on a long sequence started last (the host sorts by its bounds of the lengths)
+  const int zb = blockIdx.z / halves;
+  const int h = blockIdx.x, sp = blockIdx.y, b = a.rows.B <= ATTN_MAX_SEQS ? (int)a.order[zb] : zb, half = blockIdx.z % halves;
   const int row0 = half * AU_ROWS;
   const int H = a.H, kvh = h / (H / a.g.n_kv_heads);
   const int ncl = (int)gridDim.y;                              // key splits = the cluster; split sp owns tiles sp, sp + ncl, ...

@@ -707,6 +707,14 @@ int launch_attention_tc(spec_ctx* c, const Rows& rows, int R, int l, const int* 
   if (attn_long_mode(c, R, tiles_hi * 64) && c->attn_umma && c->tm_kv_ok && D == 128) {
     // long contexts: scores and P V on tcgen05, a CTA per (head, 64 rows, key split)
     const int halves = (R + AU_ROWS - 1) / AU_ROWS;
+    if (c->B <= ATTN_MAX_SEQS) {
+      int idx[ATTN_MAX_SEQS];
+      for (int b = 0; b < c->B; ++b) idx[b] = b;
+      // (the host's current bounds, not the bounds the launch is planned for: those are the same for all)
+      const int* len = (int)c->n_hi.size() >= c->B ? c->n_hi.data() : n_hi_pass;
+      std::stable_sort(idx, idx + c->B, [&](int x, int y) { return len[x] > len[y]; });
+      for (int b = 0; b < c->B; ++b) a.order[b] = (unsigned char)idx[b];
+    }
     // the key splits of a (sequence, row half, head) are one cluster: one CTA per SM, at most a wave of them
     a.nsplit = std::max(1, std::min(std::min(c->nsplit_attn, AU_MAX_CLUSTER), (SM_SLOTS / 2) / (H * c->B * halves)));
     dim3 grid(H, a.nsplit, c->B * halves);

@@ -129,11 +129,13 @@ def test_long_context_attention_kernels_on_small_shapes(torch, T, prompt_len, um
     assert rep.steps > 0
 
 
-@pytest.mark.parametrize("umma", [1, 0])
-def test_long_context_attention_kernels_batched_ragged(torch, umma):
+@pytest.mark.parametrize("umma,wide", [(1, 1), (0, 1), (1, 0)])
+def test_long_context_attention_kernels_batched_ragged(torch, umma, wide):
     """The long-context attention kernels on a batch of four ragged sequences (17 to 530 cached positions: less
     than one 128-key tile up to several tiles with a ragged tail; sequence b's pages interleave with the others'
-    in the pool), every sequence in lock step with an oracle of its own for three steps."""
+    in the pool), every sequence in lock step with an oracle of its own for three steps. The passes have 256 rows
+    (512 in the prompt): the projections run as 128 x 256 tiles (wide = 1) or on the weight streamer (wide = 0),
+    and the glue kernels take their many-row forms on finished sums or on partial sums."""
     from oracle.decoder import OracleModel
     from oracle.spec import OracleSpecDecoder
     from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights
@@ -147,6 +149,7 @@ def test_long_context_attention_kernels_batched_ragged(torch, umma):
     model = OracleModel(cfg, w)
     gpu = SpecDecoder(cfg, upload_weights(cfg, w), tree, 530 + 40, max_batch=4, flags=B.FLAG_KEEP_LOGITS)
     gpu.set_option(B.OPT_ATTN_UMMA, umma)
+    gpu.set_option(B.OPT_WIDE_GEMM, wide)
     gpu.set_option(B.OPT_LONG_ATTN_KEYS, 1)
     oracles = {b: OracleSpecDecoder(model, tree, 530 + 40) for b in range(4)}
     reps = run_lockstep_batch(cfg, gpu, oracles, prompts, 3, TOL_BF16, TIE_GAP)
