@@ -176,13 +176,13 @@ int64_t spec_query(const spec_ctx *ctx, int32_t what);
  * after a prefill and after an option change; steps that are traced or profiled are enqueued
  * directly). Results do not depend on it. SPEC_OPT_PHASE_TIMING [0]: record an event at the five
  * phase boundaries of every step for spec_last_step_phase_ms (costs the programmatic overlap at
- * those boundaries: about 0.03 ms of a 7B step). SPEC_OPT_CLUSTER_EPILOGUE [6]: bit mask of the projections
+ * those boundaries: about 0.03 ms of a 7B step). SPEC_OPT_CLUSTER_EPILOGUE [7]: bit mask of the projections
  * that, in passes of at most 128 rows, run as thread-block clusters which add their split-K sums through
  * distributed shared memory and apply the step that follows themselves: 1 = output and down projections
  * (residual add in place), 2 = gate+up (SwiGLU, passes of at most 64 rows), 4 = q/k/v (RoPE and cache
  * store). A projection whose bit is clear leaves partial sums for a separate kernel (other summation
- * order, same rounding points). Bits 2 and 4 are on by default: on the 7B shape they shorten a step by 2%
- * and 4.4% (bit 1 lengthens it by 2%). SPEC_OPT_WIDE_GEMM [1]: passes of more than
+ * order, same rounding points). All three are on by default: on the 7B shape they shorten a step by 2.2%,
+ * 2% and 4.4%. SPEC_OPT_WIDE_GEMM [1]: passes of more than
  * 128 rows (batched verification, batched prompt processing) run their projections as whole
  * [128 weight rows] x [256 activation rows] tiles that keep a weight tile for 256 rows at a time;
  * 0 = the weight-streaming kernel, which re-reads the weights for every 128 rows.

@@ -1,15 +1,19 @@
 // Weight-streaming bf16 linear whose split-K partial sums never leave the chip: the CTAs that
-// share an output tile form a thread-block cluster, leave their float32 accumulators in their own
-// shared memory and add them up through distributed shared memory, so the kernel writes finished
-// results and the element-wise step that used to follow in a kernel of its own runs in the epilogue.
+// share an output tile form a thread-block cluster and exchange their float32 accumulators through
+// distributed shared memory, so the kernel writes finished results and the element-wise step that
+// used to follow in a kernel of its own runs in the epilogue. The residual and SwiGLU modes push: once
+// every CTA's MMAs are complete (first cluster barrier; every ring is free then) a thread sends the
+// values of its weight row with remote stores, which nobody waits for, into the shared memory of the
+// CTA that finishes that column; after the second barrier each CTA reads only its own shared memory.
+// (Reading the parts out of the other CTAs' shared memory instead cost 3 us more per kernel.)
 //
-// Two modes (operands swapped as in gemm_stream: 128 weight rows are the MMA's M, the MT activation
+// Three modes (operands swapped as in gemm_stream: 128 weight rows are the MMA's M, the MT activation
 // rows its N; MT covers all rows of the pass):
 //  * GC_RESIDUAL (output and down projections): a cluster of 8 CTAs per 128-row weight tile, CTA r
-//    streaming the r-th eighth of the K chunks. After the cluster barrier CTA r owns output columns
-//    [16 r, 16 r + 16) of the tile: it adds the eight partial sums in rank order, adds the residual
-//    stream x in place and leaves the sum of squares of its piece of every row (the RMSNorm that
-//    follows needs the row's mean square) in ss_part[m][tile * 8 + r].
+//    streaming the r-th eighth of the K chunks. CTA r owns output columns [16 r, 16 r + 16) of the
+//    tile: it adds the eight parts in rank order, adds the residual stream x in place (old values
+//    fetched during the exchange) and leaves the sum of squares of its piece of every row (the RMSNorm
+//    that follows needs the row's mean square) in ss_part[m][tile * 8 + r].
 //  * GC_SWIGLU (gate and up projections): a cluster of 3 CTAs per pair (gate tile t, up tile t); the
 //    2 KC units of the pair are cut into three equal runs, so CTA 0 holds a gate part, CTA 1 a gate
 //    and an up part (two accumulators) and CTA 2 an up part. Once every CTA's MMAs are complete (first
@@ -287,7 +291,7 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
     const int q = warp & 3;
     pdl_wait();
     if (MODE == GC_ROPE) rope_meta();
-    if (MODE == GC_SWIGLU) {
+    if (MODE == GC_SWIGLU || MODE == GC_RESIDUAL) {
       // the accumulators stay in tensor memory until every CTA of the cluster has finished its MMAs (below)
       if (n_units > 0) mbar_wait(acc_full, 0, p.status, 32);
     } else if (n_units > 0 && mbar_wait(acc_full, 0, p.status, 32)) {
@@ -321,6 +325,84 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
   // MMAs are complete, so every ring is free) ----
   __syncwarp();
   cluster_sync_all();
+
+  if (MODE == GC_RESIDUAL) {
+    // Pushed like the gate+up parts below: a thread sends the MT values of its weight row w into the shared memory
+    // of the CTA that finishes column w (CTA w / 16), buffer [source CTA][activation row][16 columns]; after the
+    // second barrier CTA `rank` adds the eight parts of its columns [16 rank, +16) in rank order, adds the residual
+    // stream in place (its old values were fetched during the exchange) and leaves the sums of squares.
+    constexpr int CP = 16;
+    static_assert(CS * MT * CP * 4 <= Cfg::RING_BYTES, "the parts of a CTA's columns must fit the ring");
+    constexpr int ITEMS = MT * 4, PER = (ITEMS + 127) / 128;   // (row m, group of four columns c4)
+    const int e = threadIdx.x - 64;
+    const bool fin = warp >= 2 && n_units > 0;
+    float4 xo[PER];
+    bool on[PER];
+    if (fin) {
+#pragma unroll
+      for (int k = 0; k < PER; ++k) {
+        const int it = e + 128 * k, m = it >> 2, c4 = it & 3;
+        const int col = t * 128 + rank * 16 + c4 * 4;
+        on[k] = it < ITEMS && m < p.M && col < p.N;
+        xo[k] = on[k] ? *reinterpret_cast<const float4*>(p.x + (size_t)m * p.N + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      const int q = warp & 3, w = q * 32 + lane;
+      const uint32_t dst = dsmem_addr(smem_u32(staging), (uint32_t)(w >> 4)) + (uint32_t)((rank * MT * CP + (w & 15)) * 4);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      tc_fence_after();
+      if (MT >= 32) {
+#pragma unroll
+        for (int g = 0; g < MT / 32; ++g) {
+          uint32_t r[32];
+          tmem_ld32(taddr + g * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) dsmem_st(dst + (uint32_t)((g * 32 + j) * CP * 4), __uint_as_float(r[j]));
+        }
+      } else {
+        uint32_t r[16];
+        tmem_ld16(taddr, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dsmem_st(dst + (uint32_t)(j * CP * 4), __uint_as_float(r[j]));
+      }
+      tc_fence_before();
+    }
+    __syncwarp();
+    cluster_sync_all();                                       // the parts have arrived (release / acquire)
+    if (fin) {
+      float ss[PER];
+#pragma unroll
+      for (int k = 0; k < PER; ++k) {
+        const int it = e + 128 * k, m = it >> 2, c4 = it & 3;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (it < ITEMS) {
+          const float* src = staging + m * CP + c4 * 4;
+#pragma unroll
+          for (int rr = 0; rr < CS; ++rr) add4(acc, *reinterpret_cast<const float4*>(src + rr * MT * CP));   // rank order
+        }
+        add4(xo[k], acc);
+        ss[k] = xo[k].x * xo[k].x + xo[k].y * xo[k].y + xo[k].z * xo[k].z + xo[k].w * xo[k].w;
+        if (on[k]) *reinterpret_cast<float4*>(p.x + (size_t)m * p.N + t * 128 + rank * 16 + c4 * 4) = xo[k];
+      }
+      if (p.ss_part) {
+        // the four column groups of a row sit in four neighbouring lanes
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+          float v = on[k] ? ss[k] : 0.f;
+          v += __shfl_xor_sync(0xffffffffu, v, 1);
+          v += __shfl_xor_sync(0xffffffffu, v, 2);
+          const int it = e + 128 * k, m = it >> 2;
+          if ((it & 3) == 0 && it < ITEMS && m < p.M)
+            p.ss_part[(size_t)m * (((p.N + 127) >> 7) * CS) + t * CS + rank] = v;
+        }
+      }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+    return;
+  }
 
   if (MODE == GC_SWIGLU) {
     // Push instead of pull: a thread owns weight row w of its CTA's accumulators and sends its MT values
@@ -395,53 +477,7 @@ gemm_cluster(const __grid_constant__ StreamTmaps tm, const ClusterGemmParams p) 
     // uses the first one: the step costs about one round trip, not one per item.
     const int e = threadIdx.x - 64;                        // 0..127
     const uint32_t stage_local = smem_u32(staging);
-    if (MODE == GC_RESIDUAL) {
-      // CTA `rank` finishes output columns [16 rank, +16) of the tile for every activation row: items
-      // (row m, group of four columns c4), a warp reading whole 64-byte pieces of staged rows
-      constexpr int ITEMS = MT * 4, PER = (ITEMS + 127) / 128;
-      float4 xo[PER], acc[PER];
-      bool on[PER];
-#pragma unroll
-      for (int k = 0; k < PER; ++k) {
-        const int it = e + 128 * k, m = it >> 2, c4 = it & 3;
-        const int col = t * 128 + rank * 16 + c4 * 4;
-        on[k] = it < ITEMS && m < p.M && col < p.N;
-        xo[k] = on[k] ? *reinterpret_cast<const float4*>(p.x + (size_t)m * p.N + col) : make_float4(0.f, 0.f, 0.f, 0.f);
-        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-#pragma unroll
-      for (int rr = 0; rr < CS; ++rr) {
-        const uint32_t base = dsmem_addr(stage_local, (uint32_t)rr);
-        float4 v[PER];
-#pragma unroll
-        for (int k = 0; k < PER; ++k) {
-          const int it = e + 128 * k, m = it >> 2, c4 = it & 3;
-          v[k] = it < ITEMS ? dsmem_ld4(base + (uint32_t)((m * Cfg::PITCH + rank * 16 + c4 * 4) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int k = 0; k < PER; ++k) add4(acc[k], v[k]);      // rank order: the same sum whoever computes it
-      }
-      float ss[PER];
-#pragma unroll
-      for (int k = 0; k < PER; ++k) {
-        const int it = e + 128 * k, m = it >> 2, c4 = it & 3;
-        add4(xo[k], acc[k]);
-        ss[k] = xo[k].x * xo[k].x + xo[k].y * xo[k].y + xo[k].z * xo[k].z + xo[k].w * xo[k].w;
-        if (on[k]) *reinterpret_cast<float4*>(p.x + (size_t)m * p.N + t * 128 + rank * 16 + c4 * 4) = xo[k];
-      }
-      if (p.ss_part) {
-        // the four column groups of a row sit in four neighbouring lanes
-#pragma unroll
-        for (int k = 0; k < PER; ++k) {
-          float v = on[k] ? ss[k] : 0.f;
-          v += __shfl_xor_sync(0xffffffffu, v, 1);
-          v += __shfl_xor_sync(0xffffffffu, v, 2);
-          const int it = e + 128 * k, m = it >> 2;
-          if ((it & 3) == 0 && it < ITEMS && m < p.M)
-            p.ss_part[(size_t)m * (((p.N + 127) >> 7) * CS) + t * CS + rank] = v;
-        }
-      }
-    } else if (MODE == GC_ROPE) {
+    if (MODE == GC_ROPE) {
       // the tile holds 128 / D whole heads. CTA `rank` takes the activation rows rank, rank + cluster size, ...; an item is
       // (row, group of four rotation pairs): columns [lo, lo + 4) and [lo + D/2, lo + D/2 + 4) of one head
       constexpr int ITEMS = R_ITEMS, PER = R_PER;

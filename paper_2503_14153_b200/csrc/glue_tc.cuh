@@ -151,6 +151,58 @@ norm_reduce_tc(float* __restrict__ x, const PartView pv, const float* __restrict
     emit(c4, *reinterpret_cast<const float4*>(xr + c4 * 4), *reinterpret_cast<const float4*>(gain + c4 * 4));
 }
 
+// RMSNorm of rows whose sums of squares already exist in pieces (the residual cluster epilogue leaves
+// ss_part[m][n_ss], the sum of squares of every 16-column piece of row m): u[m] = bf16(x / rms(x) * g).
+// gridDim.y plain CTAs share a row, each adding all the row's pieces itself in a fixed order (the same sum in
+// every CTA), so nothing is exchanged between CTAs. One trip to L2 per thread.
+__global__ void __launch_bounds__(NORM_THREADS)
+norm_scaled_tc(const float* __restrict__ x, const float* __restrict__ ss_part, int n_ss, const float* __restrict__ gain,
+               float eps, bf16* __restrict__ u, float* __restrict__ hid, int d, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  const int m = blockIdx.x;
+  const float* xr = x + (size_t)m * d;
+  const int n4 = d >> 2;
+  const int per = (n4 + (int)gridDim.y - 1) / (int)gridDim.y;
+  const int c_lo = blockIdx.y * per, c_hi = min(n4, c_lo + per);
+  float4 gk[NORM_CACHE];
+#pragma unroll
+  for (int k = 0; k < NORM_CACHE; ++k) {
+    const int c4 = c_lo + threadIdx.x + k * NORM_THREADS;
+    gk[k] = c4 < c_hi ? *reinterpret_cast<const float4*>(gain + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  float4 keep[NORM_CACHE];
+#pragma unroll
+  for (int k = 0; k < NORM_CACHE; ++k) {
+    const int c4 = c_lo + threadIdx.x + k * NORM_THREADS;
+    keep[k] = c4 < c_hi ? *reinterpret_cast<const float4*>(xr + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < n_ss; i += NORM_THREADS) ss += __ldcg(ss_part + (size_t)m * n_ss + i);
+  __shared__ float red[NORM_THREADS / 32];
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < NORM_THREADS / 32; ++w) tot += red[w];
+  const float inv = rsqrtf(tot / (float)d + eps);
+  auto emit = [&](int c4, const float4& v, const float4& g) {
+    const float4 o = make_float4(v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
+    *reinterpret_cast<uint2*>(u + (size_t)m * d + c4 * 4) = pack4_bf16(o.x, o.y, o.z, o.w);
+    if (hid) *reinterpret_cast<float4*>(hid + (size_t)m * d + c4 * 4) = o;
+  };
+#pragma unroll
+  for (int k = 0; k < NORM_CACHE; ++k) {
+    const int c4 = c_lo + threadIdx.x + k * NORM_THREADS;
+    if (c4 < c_hi) emit(c4, keep[k], gk[k]);
+  }
+  for (int c4 = c_lo + threadIdx.x + NORM_CACHE * NORM_THREADS; c4 < c_hi; c4 += NORM_THREADS)
+    emit(c4, *reinterpret_cast<const float4*>(xr + c4 * 4), *reinterpret_cast<const float4*>(gain + c4 * 4));
+}
+
 // The same operation for passes of many rows (batched verification, prompt processing): one CTA of
 // NORMW_THREADS per row, no cluster. With hundreds of rows the kernel is bound by bandwidth, not by the
 // latency of one row, so what counts is loads in flight: a thread fetches all its pieces of x and of the

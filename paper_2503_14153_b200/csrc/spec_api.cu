@@ -207,7 +207,7 @@ struct spec_ctx {
   CUtensorMap tm_kv;                   // 5-D view of the page pool for its TMA loads
   bool tm_kv_ok = false;
   bool wide_gemm = true;               // SPEC_OPT_WIDE_GEMM: passes of more than 128 rows use the 128 x 256-tile kernel
-  int cluster_epilogue = 6;            // SPEC_OPT_CLUSTER_EPILOGUE: which projections finish their split-K sums inside a cluster
+  int cluster_epilogue = 7;            // SPEC_OPT_CLUSTER_EPILOGUE: which projections finish their split-K sums inside a cluster
                                        // (bits: 1 output/down, 2 gate+up, 4 q/k/v; measured on the 7B shape: only gate+up pays)
   int small_gemm_ctas = 288;           // CTAs of GEMMs with at most 48 weight tiles (Wo, down); 288 since the weights are pre-tiled (192 before)
   std::vector<int> h_parent, h_depth, h_rank;
@@ -224,6 +224,7 @@ struct spec_ctx {
   uint32_t *d_anc_tree, *d_anc_chain;
   const void **d_mw, **d_mb;
   float *d_x, *d_hid, *d_h_last, *d_part, *d_logits, *d_pval, *d_part_o, *d_part_ml, *d_pk_val;
+  float* d_ss_part = nullptr;          // [128 rows][d / 128 tiles x 8]: sums of squares the residual cluster epilogue leaves
   float2* d_rope;
   void *d_u, *d_q, *d_attn, *d_act, *d_hq, *d_hq_last, *d_r, *d_pool;
   size_t part_floats;
@@ -397,6 +398,7 @@ size_t carve(spec_ctx* c, void* base) {
   c->d_pval = b.take<float>((size_t)c->ntile_lm * M, 1024); c->d_pidx = b.take<int>((size_t)c->ntile_lm * M, 1024);
   c->d_part_o = c->tc ? b.take<float>((size_t)c->nsplit_attn * M * HD, 1024) : nullptr;
   c->d_part_ml = c->tc ? b.take<float>((size_t)c->nsplit_attn * M * f.n_heads * 2) : nullptr;
+  c->d_ss_part = c->tc ? b.take<float>((size_t)128 * ((d + 127) / 128) * GC_RES_CLUSTER) : nullptr;
   c->d_pk_val = b.take<float>((size_t)c->topk_blocks * B * (K ? K : 1) * c->kmax);
   c->d_pk_idx = b.take<int>((size_t)c->topk_blocks * B * (K ? K : 1) * c->kmax);
   c->d_rope = b.take<float2>((size_t)c->cap * (f.head_dim / 2));
@@ -606,7 +608,7 @@ int run_gemm_cluster(spec_ctx* c, int mode, const void* in, int M, int K, const 
   const CUtensorMap* tb = c->tmap(in, std::max<size_t>(round_up(M, 16), MT), K, MT);
   if (!tb) return c->fail(SPEC_E_CUDA, "cuTensorMapEncodeTiled failed (activations)");
   tm.b = *tb;
-  p.x = x; p.ss_part = nullptr; p.act = act_out; p.status = c->d_status;
+  p.x = x; p.ss_part = mode == GC_RESIDUAL ? c->d_ss_part : nullptr; p.act = act_out; p.status = c->d_status;
   int n_tiles = (N + 127) / 128;
   if (mode == GC_ROPE) {
     const int tq = (HD + 127) / 128, tk = (KD + 127) / 128;
@@ -819,8 +821,13 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, cons
   const int kp0 = (HD + 127) / 128 * 128, vp0 = kp0 + (KD + 127) / 128 * 128;   // padded columns of k and v in the QKV partials
   const int up0 = (F + 127) / 128 * 128;                                        // and of the up projection
   // (passes of more than 128 rows are bound by bandwidth, not by a row's latency: one plain CTA per row)
+  // (after a residual cluster epilogue the pieces' sums of squares exist already: ss_ready)
+  bool ss_ready = false;
+  const int n_ss = ((d + 127) / 128) * GC_RES_CLUSTER;
 #define NORM_LAUNCH(pv, gain, uq, hid)                                                                   \
-  if (M > 128) {                                                                                         \
+  if (ss_ready && M <= 128) {                                                                            \
+    KLAUNCH("norm_reduce_tc", norm_scaled_tc, dim3(M, NORM_CLUSTER), dim3(NORM_THREADS), 0, (const float*)c->d_x, (const float*)c->d_ss_part, n_ss, gain, f.rms_eps, uq, hid, d); \
+  } else if (M > 128) {                                                                                         \
     KLAUNCH("norm_reduce_tc", norm_rows_wide, dim3(M), dim3(NORMW_THREADS), 0, c->d_x, pv, gain, f.rms_eps, uq, hid, d); \
   } else {                                                                                               \
     KLAUNCH("norm_reduce_tc", norm_reduce_tc, dim3(M, NORM_CLUSTER), dim3(NORM_THREADS), 0, c->d_x, pv, gain, f.rms_eps, uq, hid, d); \
@@ -850,7 +857,11 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, cons
       if (cluster_gemm_ok(c, GC_RESIDUAL, M, HD)) {
         // the cluster adds its split-K sums and the residual stream itself: nothing left for the norm kernel to add
         if ((r = run_gemm_cluster(c, GC_RESIDUAL, c->d_attn, M, HD, mats, d, c->d_x, nullptr, SPEC_PROFILE_WO))) return r;
-      } else if ((r = run_gemm(c, c->d_attn, M, HD, 1, mats, rws, SPEC_PROFILE_WO, &vo))) return r;
+        ss_ready = true;
+      } else {
+        ss_ready = false;
+        if ((r = run_gemm(c, c->d_attn, M, HD, 1, mats, rws, SPEC_PROFILE_WO, &vo))) return r;
+      }
     }
     NORM_LAUNCH(vo, c->fn[l], u, (float*)nullptr);
     {
@@ -872,7 +883,11 @@ int forward_layers_tc(spec_ctx* c, int R, bool chain, const int* n_hi_pass, cons
       pend = PartView{};
       if (cluster_gemm_ok(c, GC_RESIDUAL, M, F)) {
         if ((r = run_gemm_cluster(c, GC_RESIDUAL, act, M, F, mats, d, c->d_x, nullptr, SPEC_PROFILE_DOWN))) return r;
-      } else if ((r = run_gemm(c, act, M, F, 1, mats, rws, SPEC_PROFILE_DOWN, &pend))) return r;
+        ss_ready = true;
+      } else {
+        ss_ready = false;
+        if ((r = run_gemm(c, act, M, F, 1, mats, rws, SPEC_PROFILE_DOWN, &pend))) return r;
+      }
     }
   }
   NORM_LAUNCH(pend, c->final_norm, static_cast<bf16*>(c->d_hq), c->d_hid);
