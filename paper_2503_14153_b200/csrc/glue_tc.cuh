@@ -482,9 +482,13 @@ topk_slices(const float* __restrict__ logits, int V, int rows_total, int slice, 
 
 // lm_head consumers of the GEMM's partial sums. argmax_partials_tc: row m, vocabulary slice
 // blockIdx.y of gridDim.y: logits = sum of the slots (written out when `logits` is given), the
-// slice's best (value desc, index asc) goes to pval / pidx [m][gridDim.y].
+// slice's best (value desc, index asc) goes to pval / pidx [m][gridDim.y]. The CTA of a row that
+// arrives last (arrive[m], zero between launches) picks the row's best among the slices' and writes
+// pval2[m] / pidx2[m]: the order (value desc, index asc) is total, so the result does not depend on
+// who arrives last, and no finishing kernel is needed.
 __global__ void __launch_bounds__(256)
 argmax_partials_tc(const PartView pv, int V, float* __restrict__ logits, float* __restrict__ pval, int* __restrict__ pidx,
+                   unsigned int* __restrict__ arrive, float* __restrict__ pval2, int* __restrict__ pidx2,
                    unsigned long long* tr) {
   KTrace kt(tr);
   pdl_launch_dependents();
@@ -512,17 +516,43 @@ argmax_partials_tc(const PartView pv, int V, float* __restrict__ logits, float* 
   warp_argmax(bv, bi);
   if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
   __syncthreads();
+  __shared__ int last_s;
   if (threadIdx.x == 0) {
     for (int w = 1; w < (int)(blockDim.x >> 5); ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
     pval[(size_t)m * nsl + blockIdx.y] = bv;
     pidx[(size_t)m * nsl + blockIdx.y] = bi;
+    __threadfence();
+    const unsigned int old = atomicAdd(arrive + m, 1u);
+    last_s = old == (unsigned int)(nsl - 1);
+    if (last_s) arrive[m] = 0u;
+  }
+  __syncthreads();
+  if (!last_s) return;
+  __threadfence();
+  bv = -INFINITY; bi = 0x7fffffff;
+  for (int t = threadIdx.x; t < nsl; t += blockDim.x) {
+    const float v = __ldcg(pval + (size_t)m * nsl + t); const int i = __ldcg(pidx + (size_t)m * nsl + t);
+    if (better(v, i, bv, bi)) { bv = v; bi = i; }
+  }
+  __syncthreads();                                           // sv / si are reused
+  warp_argmax(bv, bi);
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
+    pval2[m] = bv;
+    pidx2[m] = bi;
   }
 }
 
-// topk_slices over the partial sums of the heads' lm_head GEMM instead of materialised logits.
+// topk_slices over the partial sums of the heads' lm_head GEMM instead of materialised logits. The CTA of a
+// row that arrives last (arrive[row], zero between launches) merges the row's lists itself (topk_merge_row:
+// the result does not depend on who that is). Dynamic shared memory: the larger of slice * 4 and
+// gridDim.x * kmax * 8 bytes.
 __global__ void __launch_bounds__(256)
-topk_slices_tc(const PartView pv, int V, int rows_total, int slice, int kmax, float* __restrict__ pk_val,
-               int* __restrict__ pk_idx, unsigned long long* tr) {
+topk_slices_tc(const PartView pv, int V, int rows_total, int slice, int kmax, float* pk_val, int* pk_idx,
+               unsigned int* __restrict__ arrive, int K, const int* __restrict__ root_tok,
+               const int* __restrict__ cand_override, int* __restrict__ cand, unsigned long long* tr) {
   KTrace kt(tr);
   pdl_launch_dependents();
   pdl_wait();
@@ -552,33 +582,17 @@ topk_slices_tc(const PartView pv, int V, int rows_total, int slice, int kmax, fl
     }
     __syncthreads();
   }
-}
-
-// Finishes the per-row argmax from the per-(tile, lane quarter) partials of the lm_head
-// epilogue: one CTA per row, result in pval2[m] / pidx2[m].
-__global__ void __launch_bounds__(256)
-argmax_finish(const float* __restrict__ pval, const int* __restrict__ pidx, int ntile, float* __restrict__ pval2,
-              int* __restrict__ pidx2, unsigned long long* tr) {
-  KTrace kt(tr);
-  pdl_launch_dependents();
-  pdl_wait();
-  if (threadIdx.x == 0) trace_mark_min(tr, 2);
-  const int m = blockIdx.x;
-  float bv = -INFINITY; int bi = 0x7fffffff;
-  for (int t = threadIdx.x; t < ntile; t += blockDim.x) {
-    const float v = pval[(size_t)m * ntile + t]; const int i = pidx[(size_t)m * ntile + t];
-    if (better(v, i, bv, bi)) { bv = v; bi = i; }
-  }
-  __shared__ float sv[8];
-  __shared__ int si[8];
-  warp_argmax(bv, bi);
-  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
-  __syncthreads();
+  __shared__ int last_s;
   if (threadIdx.x == 0) {
-    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
-    pval2[m] = bv;
-    pidx2[m] = bi;
+    __threadfence();
+    const unsigned int old = atomicAdd(arrive + row, 1u);
+    last_s = old == gridDim.x - 1;
+    if (last_s) arrive[row] = 0u;
   }
+  __syncthreads();
+  if (!last_s) return;
+  __threadfence();
+  topk_merge_row(pk_val, pk_idx, (int)gridDim.x, row, K, kmax, root_tok, cand_override, cand, zs);
 }
 
 // y[m][n] = sum of the partial slots (logical columns of a single matrix): the stand-alone linear.

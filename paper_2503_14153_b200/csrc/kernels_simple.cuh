@@ -750,30 +750,25 @@ __global__ void medusa_lmhead_topk(const T* __restrict__ r, const T* __restrict_
 }
 
 // Merges the partial lists of one (sequence, head) row into cand[b][k+1][0..kmax) and applies
-// the optional override table; block 0 of each sequence also writes cand[b][0][0] = root.
-// The row's nblocks * kmax candidates sit in shared memory, every thread looking after each
-// blockDim-th of them; kmax rounds of a block-wide argmax (value desc, index asc), the owner of
-// the winner taking it out. Dynamic shared memory: nblocks * kmax * 8 bytes. At most 8 warps.
-__global__ void __launch_bounds__(256)
-topk_merge(const float* __restrict__ pk_val, const int* __restrict__ pk_idx, int nblocks,
-           int rows_total, int K, int kmax, const int* __restrict__ root_tok,
-           const int* __restrict__ cand_override, int* __restrict__ cand, unsigned long long* tr) {
-  KTrace kt(tr);
-  pdl_launch_dependents();
-  pdl_wait();
-  if (threadIdx.x == 0) trace_mark_min(tr, 2);
-  extern __shared__ float ms[];     // values [nblocks*kmax], indices [nblocks*kmax]
+// the optional override table; the row of head 0 of each sequence also writes cand[b][0][0] = root.
+// The row's nblocks * kmax candidates sit in shared memory (ms: nblocks * kmax * 8 bytes), every
+// thread looking after each blockDim-th of them; kmax rounds of a block-wide argmax (value desc,
+// index asc), the owner of the winner taking it out. Called by all threads of a CTA of at most 8
+// warps; the lists are read around L1 (another CTA of the same launch may have written them).
+__device__ __forceinline__ void topk_merge_row(const float* pk_val, const int* pk_idx, int nblocks, int row, int K, int kmax,
+                                               const int* __restrict__ root_tok, const int* __restrict__ cand_override,
+                                               int* __restrict__ cand, float* ms) {
   __shared__ float wv[8];
   __shared__ int wi[8], wc[8];
-  const int row = blockIdx.x, b = row / K, k = row % K;
+  const int b = row / K, k = row % K;
   const int total = nblocks * kmax;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
   float* v = ms;
   int* ix = reinterpret_cast<int*>(ms + total);
   for (int c = threadIdx.x; c < total; c += blockDim.x) {
     const size_t o = (size_t)row * total + c;          // lists of a row are contiguous: [row][block][kmax]
-    v[c] = pk_val[o];
-    ix[c] = pk_idx[o];
+    v[c] = __ldcg(pk_val + o);
+    ix[c] = __ldcg(pk_idx + o);
   }
   // the override entries do not depend on the lists: one load per round, issued up front
   int ovr = -1;
@@ -804,6 +799,19 @@ topk_merge(const float* __restrict__ pk_val, const int* __restrict__ pk_idx, int
     __syncthreads();
   }
   if (k == 0 && threadIdx.x == 0) cand[(size_t)b * (K + 1) * kmax] = root_tok[b];
+}
+
+// The merge as a kernel of its own (one CTA per row; dynamic shared memory nblocks * kmax * 8 bytes).
+__global__ void __launch_bounds__(256)
+topk_merge(const float* __restrict__ pk_val, const int* __restrict__ pk_idx, int nblocks,
+           int rows_total, int K, int kmax, const int* __restrict__ root_tok,
+           const int* __restrict__ cand_override, int* __restrict__ cand, unsigned long long* tr) {
+  KTrace kt(tr);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x == 0) trace_mark_min(tr, 2);
+  extern __shared__ float ms[];     // values [nblocks*kmax], indices [nblocks*kmax]
+  topk_merge_row(pk_val, pk_idx, nblocks, blockIdx.x, K, kmax, root_tok, cand_override, cand, ms);
 }
 
 }  // namespace spec

@@ -234,6 +234,7 @@ struct spec_ctx {
   bool trace_on = false;
   unsigned long long* d_trace = nullptr;
   unsigned int* d_attn_arrive = nullptr;
+  unsigned int* d_row_arrive = nullptr;   // [Mcap] arrival counters of the per-row finishing steps, zero between launches
   float* d_pval2 = nullptr;            // finished per-row argmax (tensor-core path)
   int* d_pidx2 = nullptr;
   int trace_n = 0;
@@ -355,6 +356,7 @@ size_t carve(spec_ctx* c, void* base) {
   c->d_status = b.take<int>(4);
   c->d_trace = b.take<unsigned long long>((size_t)TRACE_CAP * 4);
   c->d_attn_arrive = b.take<unsigned int>((size_t)B * f.n_heads * 2);
+  c->d_row_arrive = b.take<unsigned int>(c->Mcap);
   c->d_pval2 = b.take<float>(c->Mcap); c->d_pidx2 = b.take<int>(c->Mcap);
   c->d_draws = b.take<int>(B);
   c->d_n = b.take<int>(B); c->d_cnt = b.take<int>(B); c->d_n_old = b.take<int>(B); c->d_root = b.take<int>(B);
@@ -968,11 +970,11 @@ int heads_tc(spec_ctx* c, const int* ov) {
     int r = run_gemm(c, c->d_r, rows_total, d, 1, mats, rws, SPEC_PROFILE_OFF, &pl);
     if (r) return r;
   }
-  KLAUNCH("topk_slices_tc", topk_slices_tc, dim3(c->topk_blocks, rows_total), dim3(256), (size_t)c->topk_slice * sizeof(float),
-          pl, f.vocab, rows_total, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx);
-  size_t sm2 = (size_t)c->topk_blocks * kmax * 8 + (size_t)c->topk_blocks * 4;
-  KLAUNCH("topk_merge", topk_merge, dim3(rows_total), dim3(256), sm2, (const float*)c->d_pk_val, (const int*)c->d_pk_idx,
-          c->topk_blocks, rows_total, K, kmax, (const int*)c->d_root, ov, c->d_cand);
+  // the row's last-arriving CTA merges the slices' lists: no merge kernel
+  const size_t sm_topk = std::max((size_t)c->topk_slice * sizeof(float), (size_t)c->topk_blocks * kmax * 8);
+  if (sm_topk > 48 * 1024) return c->fail(SPEC_E_BADARG, "top-k lists do not fit the merge's shared memory");
+  KLAUNCH("topk_slices_tc", topk_slices_tc, dim3(c->topk_blocks, rows_total), dim3(256), sm_topk,
+          pl, f.vocab, rows_total, c->topk_slice, kmax, c->d_pk_val, c->d_pk_idx, c->d_row_arrive, K, (const int*)c->d_root, ov, c->d_cand);
   return SPEC_OK;
 }
 
@@ -988,9 +990,7 @@ int lm_head_argmax(spec_ctx* c, const T* src, int M) {
     if (r) return r;
     const int NSL = c->ntile_lm;
     KLAUNCH("argmax_partials_tc", argmax_partials_tc, dim3(M, NSL), dim3(256), 0, pl, f.vocab,
-            c->keep_logits ? c->d_logits : (float*)nullptr, c->d_pval, c->d_pidx);
-    KLAUNCH("argmax_finish", argmax_finish, dim3(M), dim3(256), 0, (const float*)c->d_pval, (const int*)c->d_pidx, NSL,
-            c->d_pval2, c->d_pidx2);
+            c->keep_logits ? c->d_logits : (float*)nullptr, c->d_pval, c->d_pidx, c->d_row_arrive, c->d_pval2, c->d_pidx2);
   } else {
     int r = linear_simple<T>(c, src, f.d_model, static_cast<const T*>(c->lm_head), c->d_logits, f.vocab, M, f.vocab, f.d_model);
     if (r) return r;
@@ -1362,6 +1362,7 @@ int spec_create(const spec_config* cfg, const spec_weights* w, const spec_tree* 
   up(c->d_mb, c->mb.data(), c->mb.size() * sizeof(void*));
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 4 * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_attn_arrive, 0, (size_t)cfg->max_batch * cfg->n_heads * 2 * sizeof(unsigned int), c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_row_arrive, 0, (size_t)c->Mcap * sizeof(unsigned int), c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_cand, 0, (size_t)cfg->max_batch * (c->K + 1) * c->kmax * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) { g_create_error = std::string("set-up copies: ") + cudaGetErrorString(e); delete c; return SPEC_E_CUDA; }
