@@ -60,21 +60,21 @@ def test_c1_7b_width_depth_curve_vs_oracle(torch, c1_weights_16_layers, layers):
 
 
 def test_c1_7b_width_8_layers_prompt_256_multi_step_vs_oracle(torch, c1_weights_16_layers):
-    """The 7B kernels on the benchmark's prompt length and tree (256 tokens, T = 64) at 8 layers: at least 24
+    """The 7B kernels on the benchmark's prompt length and tree (256 tokens, T = 64) at 8 layers: at least 32
     emitted tokens in lock step with the oracle."""
     from paper_2503_14153_b200 import build_tree
     from tests_lockstep import run_lockstep
     cfg = get_config("c1", n_layers=8)
     w = {k: v for k, v in c1_weights_16_layers.items() if not k.startswith("layers.") or int(k.split(".")[1]) < 8}
     tree = build_tree(cfg.topk, cfg.tree_nodes)
-    # (the row error has a tail: the worst of the ~1600 rows of 25 steps was measured at 2.7% of the row's largest
+    # (the row error has a tail: the worst of the ~2000 rows of 32 steps was measured at 2.7% of the row's largest
     # value, against 1.7% for the worst of the 64 rows of the depth curve's single step; the bound here is the
     # stated 2e-2 times that ratio, with a margin)
-    rep = run_lockstep(cfg, w, tree, draw_prompt(cfg), 24, 3.5e-2, TIE_GAP, check_kv_every=8, tie_from_row_error=True)
+    rep = run_lockstep(cfg, w, tree, draw_prompt(cfg), 32, 3.5e-2, TIE_GAP, check_kv_every=8, tie_from_row_error=True)
     print(f"8 layers, prompt 256: {rep.steps} steps, {len(rep.tokens)} tokens, logits rel err {rep.max_logit_err:.4f}, hidden "
           f"{rep.max_hidden_err:.4f}, cache {rep.max_kv_err:.4f}, near ties {len(rep.near_ties)} of {rep.decisions} decisions, "
           f"largest excused gap {max([t[2] for t in rep.near_ties], default=0.0):.4f}")
-    assert len(rep.tokens) >= 24 and rep.excused_fraction < 0.10
+    assert len(rep.tokens) >= 32 and rep.excused_fraction < 0.10
 
 
 def test_c1_7b_shape_full_depth_one_step_vs_oracle(torch):
@@ -114,9 +114,9 @@ def c3_two_layers(torch):
 @pytest.mark.parametrize("T", [16, 32, 64, 128])
 def test_c3_long_context_two_layers_vs_oracle(torch, c3_two_layers, T):
     """Configuration 3 (8192 cached positions) with trees of 16, 32, 64 and 128 nodes on two layers of the
-    7B shape, two steps each against the oracle: the CTA-per-16-rows kernel at T >= 32, and at T = 16 the
-    kernel with KV splits, tiles fetched ahead of the dependency, the merge of the splits by the last CTA
-    and the tree mask at the cache's end."""
+    7B shape, two steps each against the oracle: the tcgen05 attention with its key splits merged inside a
+    cluster (one row half at T <= 64, two at T = 128; 16 and 32 valid rows of 64 at the small trees), tiles
+    fetched ahead of the dependency wait, and the tree mask at the cache's end."""
     from oracle.spec import OracleSpecDecoder
     from paper_2503_14153_b200 import SpecDecoder, build_tree
     from paper_2503_14153_b200 import binding as B
