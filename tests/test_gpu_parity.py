@@ -113,7 +113,7 @@ def test_small_bf16_d512_cluster_epilogues(torch):
 def test_long_context_attention_kernels_on_small_shapes(torch, T, prompt_len, umma):
     """The long-context attention kernels (tcgen05 scores and P V with umma = 1, the shared-K/V mma.sync kernel with
     umma = 0) forced onto short contexts by lowering their threshold to one position: one and several 128-key
-    tiles, key splits merged by the last CTA, two row halves at T = 128, trees of 16 and 32 rows, and prompt
+    tiles, key splits merged inside a cluster (umma = 1) or by the last CTA (umma = 0), idle splits, two row halves at T = 128, trees of 16 and 32 rows, and prompt
     processing in 128-row passes, all against the oracle."""
     from paper_2503_14153_b200 import SpecDecoder, build_tree, upload_weights
     from paper_2503_14153_b200 import binding as B
