@@ -19,9 +19,15 @@
 // exponentiates, the tensor cores work for the other. A producer warp brings a tile's four 16 KB slabs
 // (K / V x dims 0..63 / 64..127) with four 5-dimensional TMA loads straight out of the page pool -- the
 // library places page p of sequence b at pool page p * max_batch + b and keeps the pages of a (layer, head)
-// side by side, so a sequence's pages are a strided dimension of the tensor map --; one thread issues all MMAs. The four streams of a row (two groups x two
-// key halves) are merged through shared memory, the key splits by the CTA that arrives last. Every wait is
-// bounded.
+// side by side, so a sequence's pages are a strided dimension of the tensor map --; one thread issues all
+// MMAs. The four streams of a row (two groups x two key halves) are merged through shared memory. The key
+// splits of a (sequence, row half, head) form one thread-block cluster, split s owning tiles s, s + cluster
+// size, ... (which tiles does not depend on the length, so the first two can be asked for before the
+// dependency wait when they lie below the host's lower bound of the committed length): each CTA leaves its
+// merged partial in its own shared memory, and after a cluster barrier every CTA finishes a share of the
+// rows, reading all the partials through distributed shared memory -- no partial sums in HBM, no arrival
+// counter. Every mbarrier wait is bounded; a CTA whose wait ran out still joins the cluster barriers, so its
+// peers do not wait for it.
 #pragma once
 #include <cuda.h>
 
