@@ -446,40 +446,6 @@ medusa_act_tc(const PartView pv, int dpad, const bf16* __restrict__ hq_last, con
   }
 }
 
-// Each row's kmax best (value desc, index asc) of this block's slice of the logits go to the
-// partial lists pk_val / pk_idx [row][block][kmax]. grid (slices, rows); dynamic shared
-// memory: slice floats.
-__global__ void __launch_bounds__(256)
-topk_slices(const float* __restrict__ logits, int V, int rows_total, int slice, int kmax, float* __restrict__ pk_val,
-            int* __restrict__ pk_idx, unsigned long long* tr) {
-  KTrace kt(tr);
-  pdl_launch_dependents();
-  pdl_wait();
-  if (threadIdx.x == 0) trace_mark_min(tr, 2);
-  extern __shared__ float zs[];
-  const int row = blockIdx.y, n0 = blockIdx.x * slice, n1 = min(n0 + slice, V);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
-  for (int c = threadIdx.x; c < n1 - n0; c += blockDim.x) zs[c] = logits[(size_t)row * V + n0 + c];
-  __syncthreads();
-  __shared__ float sv[8];
-  __shared__ int si[8];
-  for (int t = 0; t < kmax; ++t) {
-    float bv = -INFINITY; int bi = 0x7fffffff;
-    for (int c = threadIdx.x; c < n1 - n0; c += blockDim.x) if (better(zs[c], n0 + c, bv, bi)) { bv = zs[c]; bi = n0 + c; }
-    warp_argmax(bv, bi);
-    if (lane == 0) { sv[warp] = bv; si[warp] = bi; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      for (int w = 1; w < nw; ++w) if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
-      const size_t o = ((size_t)row * gridDim.x + blockIdx.x) * kmax + t;
-      pk_val[o] = bv;
-      pk_idx[o] = bi;
-      if (bi != 0x7fffffff) zs[bi - n0] = -INFINITY;
-    }
-    __syncthreads();
-  }
-}
-
 // lm_head consumers of the GEMM's partial sums. argmax_partials_tc: row m, vocabulary slice
 // blockIdx.y of gridDim.y: logits = sum of the slots (written out when `logits` is given), the
 // slice's best (value desc, index asc) goes to pval / pidx [m][gridDim.y]. The CTA of a row that
@@ -545,10 +511,11 @@ argmax_partials_tc(const PartView pv, int V, float* __restrict__ logits, float* 
   }
 }
 
-// topk_slices over the partial sums of the heads' lm_head GEMM instead of materialised logits. The CTA of a
-// row that arrives last (arrive[row], zero between launches) merges the row's lists itself (topk_merge_row:
-// the result does not depend on who that is). Dynamic shared memory: the larger of slice * 4 and
-// gridDim.x * kmax * 8 bytes.
+// Per-head top-k straight from the partial sums of the heads' lm_head GEMM (no materialised logits): each
+// row's kmax best (value desc, index asc) of this block's slice of the vocabulary go to the partial lists
+// pk_val / pk_idx [row][block][kmax]; grid (slices, rows). The CTA of a row that arrives last (arrive[row],
+// zero between launches) merges the row's lists itself (topk_merge_row: the result does not depend on who
+// that is). Dynamic shared memory: the larger of slice * 4 and gridDim.x * kmax * 8 bytes.
 __global__ void __launch_bounds__(256)
 topk_slices_tc(const PartView pv, int V, int rows_total, int slice, int kmax, float* pk_val, int* pk_idx,
                unsigned int* __restrict__ arrive, int K, const int* __restrict__ root_tok,
