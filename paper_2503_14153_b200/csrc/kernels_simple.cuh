@@ -184,15 +184,6 @@ __global__ void linear_rows(const T* __restrict__ x, int ldx, const T* __restric
   }
 }
 
-// y = sum over K slices, in slice order
-__global__ void sum_partials(const float* __restrict__ part, int nsplit, size_t total, float* __restrict__ y) {
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= total) return;
-  float v = 0.f;
-  for (int s = 0; s < nsplit; ++s) v += part[(size_t)s * total + i];
-  y[i] = v;
-}
-
 // act = T(SiLU(g) * u)
 template <typename T>
 __global__ void swiglu_rows(const float* __restrict__ g, const float* __restrict__ up, T* __restrict__ act,
